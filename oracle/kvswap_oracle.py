@@ -1,0 +1,176 @@
+"""CPU oracle for the KVSwap decode hot path -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+
+A plain, slow, float64 restatement of what the paper's predictor and the sparse decode
+attention compute, one function per step, in the paper's order and notation.  It shares no
+code with the CUDA library and must never be imported by it: only the tests, the smoke
+check and the benchmark's CPU-baseline leg may call it.
+
+Notation (Sec. 4.2, Sec. 4.3, App. A.2): N cached tokens, H_q query heads, H_k = H_kv KV
+heads, d head dim, r metadata rank, A in R^{(H_k d) x r} the low-rank adapter with row block
+A_g in R^{d x r} for KV head g, g(h) = floor(h / rho) the query-head -> KV-head map with
+rho = H_q / H_kv, K_lr = Flatten(K) A the compressed K cache ("metadata"), G the group size,
+M the number of selected groups.
+
+Array conventions (all numpy, values already rounded to their storage type by the caller):
+    K, V   [B, H_kv, N, d]        q   [B, H_q, d]        proj  [H_kv, d, r]  (A_g = proj[g])
+    meta   [B, H_m, N, r]  with H_m = 1 (joint adapter, the paper's adopted design (b) of
+           Sec. 4.2) or H_m = H_kv (one adapter per KV head, design (a) of Sec. 4.2)
+    scope  "kv_head": one selection per (sequence, KV head), summing the rho query heads of
+           that KV head;  "all_heads": one selection per sequence, summing all query heads
+           (the paper's wording in Sec. 4.3, "Scoring and selection").
+
+Pins (tests/test_oracle_pins.py): every function below is checked against something other
+than itself -- exact rational arithmetic, closed forms, dense brute force, library-routine
+special cases, hand-worked examples.  The one thing that has no pin is the *quality* of the
+approximation (how much attention mass the selected groups capture): the paper prints no
+number for the predictor alone, so that statistic is only reported -- "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+_STORE = {"f32": np.float32, "f16": np.float16, "f64": np.float64}  # "f64": no rounding (pins only)
+
+
+def _rho(n_q_heads: int, n_kv_heads: int) -> int:
+    if n_q_heads % n_kv_heads:
+        raise ValueError("H_q must be a multiple of H_kv")
+    return n_q_heads // n_kv_heads
+
+
+# ------------------------------------------------------------------------------------------
+# O1  K_lr = Flatten(K) A                                                       (Sec. 4.2)
+# ------------------------------------------------------------------------------------------
+def project_keys(K: np.ndarray, proj: np.ndarray, meta_heads: int, meta_dtype: str = "f16") -> np.ndarray:
+    """Compressed K cache.  Joint: meta[b,0,n,:] = sum_g K[b,g,n,:] A_g  (Flatten is head-major,
+    column g*d+c <-> K[n,g,c]).  Per-head: meta[b,g,n,:] = K[b,g,n,:] A_g.
+    The float64 result is rounded once, to nearest-even, into the storage type."""
+    K64 = K.astype(np.float64)
+    A = proj.astype(np.float64)
+    B, Hkv, N, d = K64.shape
+    r = A.shape[2]
+    if meta_heads == 1:
+        meta = np.zeros((B, 1, N, r))
+        for g in range(Hkv):
+            meta[:, 0] += K64[:, g] @ A[g]
+    elif meta_heads == Hkv:
+        meta = np.empty((B, Hkv, N, r))
+        for g in range(Hkv):
+            meta[:, g] = K64[:, g] @ A[g]
+    else:
+        raise ValueError("meta_heads must be 1 or H_kv")
+    return meta.astype(_STORE[meta_dtype])
+
+
+# ------------------------------------------------------------------------------------------
+# O2  low-rank query  Q_h A_{g(h)}                                               (Eq. 1)
+# ------------------------------------------------------------------------------------------
+def lowrank_query(q: np.ndarray, proj: np.ndarray) -> np.ndarray:
+    q64 = q.astype(np.float64)
+    A = proj.astype(np.float64)
+    B, Hq, d = q64.shape
+    rho = _rho(Hq, A.shape[0])
+    q_lr = np.empty((B, Hq, A.shape[2]))
+    for h in range(Hq):
+        q_lr[:, h] = q64[:, h] @ A[h // rho]
+    return q_lr
+
+
+# ------------------------------------------------------------------------------------------
+# O3  per-head low-rank scores  (Q_h A_{g(h)}) K_lr^T                            (Eq. 1)
+# ------------------------------------------------------------------------------------------
+def head_scores(q_lr: np.ndarray, meta: np.ndarray, n_kv_heads: int) -> np.ndarray:
+    """s[b,h,n]; raw logits (no softmax, no 1/sqrt(d): Eq. 1 approximates Q_h K^T itself)."""
+    m64 = meta.astype(np.float64)
+    B, Hq, r = q_lr.shape
+    rho = _rho(Hq, n_kv_heads)
+    Hm = m64.shape[1]
+    s = np.empty((B, Hq, m64.shape[2]))
+    for h in range(Hq):
+        mh = 0 if Hm == 1 else h // rho
+        s[:, h] = np.einsum("br,bnr->bn", q_lr[:, h], m64[:, mh])
+    return s
+
+
+# ------------------------------------------------------------------------------------------
+# O4  one importance score per token: sum over heads      (Sec. 4.3, Scoring and selection)
+# ------------------------------------------------------------------------------------------
+def aggregate(s: np.ndarray, n_kv_heads: int, scope: str) -> np.ndarray:
+    B, Hq, N = s.shape
+    if scope == "all_heads":
+        return s.sum(axis=1, keepdims=True)
+    if scope == "kv_head":
+        rho = _rho(Hq, n_kv_heads)
+        return s.reshape(B, n_kv_heads, rho, N).sum(axis=2)
+    raise ValueError("scope must be 'kv_head' or 'all_heads'")
+
+
+# ------------------------------------------------------------------------------------------
+# O5  ReduceMax over groups of G consecutive tokens                              (Sec. 4.3)
+# ------------------------------------------------------------------------------------------
+def pool(T: np.ndarray, G: int) -> np.ndarray:
+    """R[b,s,j] = max_{0<=t<G} T[b,s,jG+t], j < floor(N/G).  The N mod G newest tokens form no
+    complete group yet (rolling buffer, Sec. 4.4.1) and get no score."""
+    B, S, N = T.shape
+    NG = N // G
+    return T[:, :, :NG * G].reshape(B, S, NG, G).max(axis=3)
+
+
+# ------------------------------------------------------------------------------------------
+# O6  TopK: the M highest-scoring groups                                         (Sec. 4.3)
+# ------------------------------------------------------------------------------------------
+def select(R: np.ndarray, M: int) -> np.ndarray:
+    """Indices of the M' = min(M, NG) largest group scores of every (b, s) problem, where of
+    two equal scores the lower index ranks first; returned sorted by index, shape [B,S,M']."""
+    B, S, NG = R.shape
+    Mp = min(M, NG)
+    idx = np.empty((B, S, Mp), dtype=np.int32)
+    for b in range(B):
+        for s in range(S):
+            order = sorted(range(NG), key=lambda j: (-R[b, s, j], j))
+            idx[b, s] = np.sort(np.asarray(order[:Mp], dtype=np.int32))
+    return idx
+
+
+def score_select(q, proj, meta, G, M, scope="kv_head"):
+    """O2..O6 chained.  Returns (idx [B,S,M'], R [B,S,NG])."""
+    Hkv = proj.shape[0]
+    R = pool(aggregate(head_scores(lowrank_query(q, proj), meta, Hkv), Hkv, scope), G)
+    return select(R, M), R
+
+
+# ------------------------------------------------------------------------------------------
+# O7  exact decode attention over the selected groups + rolling-buffer tail
+#     (Sec. 4.4 decoding; Sec. 4.4.1 rolling buffer; Sec. 4.4.4 the three sources of entries)
+# ------------------------------------------------------------------------------------------
+def attend(q, K, V, idx, G, scope="kv_head", return_probs=False):
+    """out[b,h,:] = sum_n p_n V[b,g(h),n,:],  p = softmax_n(q[b,h,:] . K[b,g(h),n,:] / sqrt(d))
+    over the token set  U_{j in idx[b,s(h)]} [jG, jG+G)  U  [floor(N/G) G, N),
+    s(h) = g(h) for scope 'kv_head', 0 for 'all_heads'.  Two-pass softmax with max subtraction.
+    Also returns lse[b,h] = log sum_n exp(logit_n)."""
+    q64, K64, V64 = q.astype(np.float64), K.astype(np.float64), V.astype(np.float64)
+    B, Hq, d = q64.shape
+    Hkv, N = K64.shape[1], K64.shape[2]
+    rho = _rho(Hq, Hkv)
+    NG = N // G
+    out = np.empty((B, Hq, d))
+    lse = np.empty((B, Hq))
+    probs = {}
+    for b in range(B):
+        for h in range(Hq):
+            g = h // rho
+            s = g if scope == "kv_head" else 0
+            tokens = [j * G + t for j in idx[b, s] for t in range(G)] + list(range(NG * G, N))
+            tokens = np.asarray(tokens, dtype=np.int64)
+            logits = (K64[b, g, tokens] @ q64[b, h]) / np.sqrt(d)
+            mx = logits.max()
+            e = np.exp(logits - mx)
+            denom = e.sum()
+            p = e / denom
+            out[b, h] = p @ V64[b, g, tokens]
+            lse[b, h] = mx + np.log(denom)
+            if return_probs:
+                probs[(b, h)] = (tokens, p)
+    if return_probs:
+        return out, lse, probs
+    return out, lse
