@@ -1,0 +1,145 @@
+/*
+ * kvswap.h -- C ABI of the KVSwap decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, on one GPU, the per-decode-step KV-entry predictor of KVSwap and
+ * the exact sparse decode attention that consumes its output:
+ *
+ *   kvswap_project_keys   K_lr = Flatten(K) A                         (Sec. 4.2)
+ *   kvswap_score_select   low-rank scores (Eq. 1) -> sum over heads -> ReduceMax over groups of
+ *                         G tokens -> TopK M groups                   (Sec. 4.3)
+ *   kvswap_sparse_decode  softmax attention over the selected groups plus the rolling-buffer
+ *                         tail                                        (Sec. 4.4, 4.4.1, 4.4.4)
+ *
+ * The paper keeps the full KV cache on disk; here it is an HBM-resident tensor and "loading a
+ * group" is a gather of G consecutive rows.
+ *
+ * Notation: B sequences, N cached tokens, H_q query heads, H_kv KV heads, rho = H_q / H_kv,
+ * g(h) = floor(h / rho), d head dim, r metadata rank, A_g = proj[g] in R^{d x r} the row block of
+ * the adapter A for KV head g, G group size, M groups to select, NG = floor(N / G).
+ * H_m ("meta_heads") is 1 for the joint-head adapter the paper adopts (design (b) of Sec. 4.2)
+ * or H_kv for one adapter per KV head (design (a)).  S is the number of selections per
+ * sequence: H_kv for KVSWAP_SCOPE_KV_HEAD (scores summed over the rho query heads of one KV
+ * head), 1 for KVSWAP_SCOPE_ALL_HEADS (scores summed over all query heads, the paper's wording).
+ *
+ * General conventions
+ *  - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *    The library never allocates, frees or keeps device memory, and never synchronises: work is
+ *    enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and the
+ *    returned status covers host-side validation and launch errors only.
+ *  - Tensors are row-major with a dense last dimension; K, V and the metadata take explicit
+ *    element strides for the leading dimensions.
+ *  - Device pointers must be 16-byte aligned, and d*sizeof(kv) and r*sizeof(meta) must be
+ *    multiples of 16 bytes (KVSWAP_ERR_ALIGN otherwise).
+ *  - Inputs must be finite.  NaN/Inf never fault but give unspecified selections/outputs.
+ *  - Errors are returned, never raised: no call aborts or traps.
+ *  - `ws` is caller-provided scratch of at least kvswap_workspace_bytes(shape) bytes.  Its
+ *    contents are undefined between calls; calls that run concurrently on different streams
+ *    need different workspaces.
+ */
+#ifndef KVSWAP_H_
+#define KVSWAP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  KVSWAP_OK = 0,
+  KVSWAP_ERR_NULL = 1,        /* a required pointer is NULL                                  */
+  KVSWAP_ERR_SHAPE = 2,       /* a size/stride/enum combination is invalid                   */
+  KVSWAP_ERR_DTYPE = 3,       /* unknown dtype tag or unsupported dtype combination          */
+  KVSWAP_ERR_ALIGN = 4,       /* pointer or row size not 16-byte aligned                     */
+  KVSWAP_ERR_WORKSPACE = 5,   /* ws_bytes smaller than kvswap_workspace_bytes()              */
+  KVSWAP_ERR_UNSUPPORTED = 6, /* valid request outside the implemented range                 */
+  KVSWAP_ERR_CUDA = 7,        /* a CUDA runtime call or kernel launch failed                 */
+  KVSWAP_ERR_INDEX = 8        /* reserved: out-of-range group index seen by a checking build */
+} kvswap_status;
+
+typedef enum { KVSWAP_F32 = 0, KVSWAP_BF16 = 1, KVSWAP_F16 = 2 } kvswap_dtype;
+typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_scope;
+
+/*
+ * Problem description shared by all calls.
+ *   kv_*   strides (in elements) of K and V, both laid out [B, H_kv, N, d];
+ *   meta_* strides (in elements) of the metadata, laid out [B, H_m, N, r].
+ * A stride of 0 means "dense": the natural stride of the contiguous tensor.
+ * Supported ranges: d in {64, 128}; r a multiple of 4 with 4 <= r <= 256; G >= 1; M >= 1;
+ * rho >= 1; G <= 1024; kv_dtype in {F32, BF16, F16}; q_dtype = kv_dtype or F32; meta_dtype in
+ * {F32, F16}.
+ */
+typedef struct {
+  int32_t batch, n_ctx, n_q_heads, n_kv_heads, head_dim; /* B, N, H_q, H_kv, d            */
+  int32_t rank, meta_heads, group_size, top_k;           /* r, H_m in {1, H_kv}, G, M     */
+  int32_t kv_dtype, meta_dtype, q_dtype, scope;          /* enums above                   */
+  int64_t kv_stride_b, kv_stride_h, kv_stride_n;
+  int64_t meta_stride_b, meta_stride_h, meta_stride_n;
+} kvswap_shape;
+
+/* Bytes of scratch any of the calls below may need for `shape`; 0 if the shape is invalid. */
+size_t kvswap_workspace_bytes(const kvswap_shape* shape);
+
+/* Validates `shape` exactly as the compute calls do (host only, touches no GPU). */
+int kvswap_validate_shape(const kvswap_shape* shape);
+
+/*
+ * Metadata build, K_lr = Flatten(K) A (Sec. 4.2), for tokens n_begin <= n < n_end (prefill: the
+ * whole context; decode: the rows of a group the rolling buffer has just completed, Sec. 4.4.1).
+ *   joint    (H_m = 1):    meta[b, 0, n, :] = sum_g K[b, g, n, :] . proj[g]   (Flatten is head-major)
+ *   per-head (H_m = H_kv): meta[b, g, n, :] =       K[b, g, n, :] . proj[g]
+ * K: [B, H_kv, N, d] kv_dtype.  proj: [H_kv, d, r] fp32, dense.  meta_out: [B, H_m, N, r]
+ * meta_dtype; fp32 accumulation, one round-to-nearest-even into meta_dtype.  Rows outside
+ * [n_begin, n_end) are not touched.  Requires 0 <= n_begin <= n_end <= N (empty range: no-op).
+ */
+int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* proj,
+                        void* meta_out, int32_t n_begin, int32_t n_end,
+                        void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Grouped critical-KV prediction (Eq. 1 and "Scoring and selection", Sec. 4.3).
+ * For every sequence b and selection scope s:
+ *   T[b,s,n] = sum_{h in scope s} (q[b,h,:] . proj[g(h)]) . meta[b, m(g(h)), n, :]   (raw logits:
+ *              no softmax, no 1/sqrt(d)),  m(g) = 0 for joint metadata, g for per-head metadata;
+ *   R[b,s,j] = max_{0<=t<G} T[b,s,jG+t]   for j < NG  (the N mod G newest tokens form no group);
+ *   the M' = min(M, NG) groups with the largest R are selected; of equal scores the lower index
+ *   wins; indices are written in ascending order.
+ * q: [B, H_q, d] q_dtype, dense (may be an approximate query, Sec. 4.3 "Online prediction").
+ * group_idx: [B, S, M] int32; entries [M', M) of each row are set to -1.
+ * n_selected: [B, S] int32, receives M'.
+ * group_scores_opt: NULL or [B, S, NG] fp32, receives R.
+ * Scores are accumulated in fp32.
+ */
+int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* proj,
+                        const void* meta, int32_t* group_idx, int32_t* n_selected,
+                        float* group_scores_opt, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Exact decode attention over the selected groups and the rolling-buffer tail (Sec. 4.4,
+ * 4.4.1, 4.4.4).  For every (b, h), with g = g(h) and row s = g (KV_HEAD) or 0 (ALL_HEADS) of
+ * the index list:
+ *   tokens  = U_{i < n_selected[b,s]} [ j_i G, j_i G + G )  U  [ NG*G, N ),  j_i = group_idx[b,s,i]
+ *   logit_n = q[b,h,:] . K[b,g,n,:] / sqrt(d)
+ *   out[b,h,:] = sum_n softmax(logit)_n V[b,g,n,:],   lse[b,h] = log sum_n exp(logit_n)
+ * computed with an fp32 online softmax in split-K partials merged by a combine pass.
+ * group_idx: [B, S, M] int32, any duplicate-free list of groups in [0, NG) (ascending order is
+ * not required); n_selected: [B, S] with 0 <= n_selected <= M.  Indices outside [0, NG) are
+ * skipped, never dereferenced.  If a head attends no token at all (n_selected = 0 and N a
+ * multiple of G) its output row is 0 and its lse is -inf.
+ * out: [B, H_q, d] fp32.  lse_opt: NULL or [B, H_q] fp32.
+ */
+int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K, const void* V,
+                         const int32_t* group_idx, const int32_t* n_selected,
+                         float* out, float* lse_opt, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Static, NUL-terminated description of a kvswap_status value. */
+const char* kvswap_status_string(int status);
+
+/* Library version as major*10000 + minor*100 + patch. */
+int kvswap_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVSWAP_H_ */

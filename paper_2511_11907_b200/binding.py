@@ -1,0 +1,130 @@
+"""ctypes binding of libkvswap.so: argument marshalling only.
+
+Every function has the name and argument order of its C entry point (include/kvswap.h).
+Tensors are torch CUDA tensors; the binding passes ``data_ptr()`` and the current CUDA stream
+and raises ``KVSwapError`` on a non-zero status.  There is no fallback: if the shared library
+is missing or cannot be loaded, importing a function from here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libkvswap.so")
+
+KVSWAP_F32, KVSWAP_BF16, KVSWAP_F16 = 0, 1, 2
+KVSWAP_SCOPE_KV_HEAD, KVSWAP_SCOPE_ALL_HEADS = 0, 1
+
+
+class KVSwapError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+class kvswap_shape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "batch", "n_ctx", "n_q_heads", "n_kv_heads", "head_dim", "rank", "meta_heads", "group_size",
+        "top_k", "kv_dtype", "meta_dtype", "q_dtype", "scope")] + [(n, ctypes.c_int64) for n in (
+        "kv_stride_b", "kv_stride_h", "kv_stride_n", "meta_stride_b", "meta_stride_h", "meta_stride_n")]
+
+    @property
+    def n_scopes(self) -> int:
+        return self.n_kv_heads if self.scope == KVSWAP_SCOPE_KV_HEAD else 1
+
+    @property
+    def n_groups(self) -> int:
+        return self.n_ctx // self.group_size
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libkvswap.so (once).  Raises if it has not been built: there is no CPU fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2511_11907_b200.build` "
+            "(the kvswap hot path has no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P, V, I32, SZ = ctypes.POINTER(kvswap_shape), ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    lib.kvswap_workspace_bytes.restype = SZ
+    lib.kvswap_workspace_bytes.argtypes = [P]
+    lib.kvswap_validate_shape.restype = ctypes.c_int
+    lib.kvswap_validate_shape.argtypes = [P]
+    lib.kvswap_project_keys.restype = ctypes.c_int
+    lib.kvswap_project_keys.argtypes = [P, V, V, V, I32, I32, V, SZ, V]
+    lib.kvswap_score_select.restype = ctypes.c_int
+    lib.kvswap_score_select.argtypes = [P, V, V, V, V, V, V, V, SZ, V]
+    lib.kvswap_sparse_decode.restype = ctypes.c_int
+    lib.kvswap_sparse_decode.argtypes = [P, V, V, V, V, V, V, V, V, SZ, V]
+    lib.kvswap_status_string.restype = ctypes.c_char_p
+    lib.kvswap_status_string.argtypes = [ctypes.c_int]
+    lib.kvswap_version.restype = ctypes.c_int
+    lib.kvswap_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().kvswap_status_string(int(status)).decode()
+
+
+def make_shape(*, batch, n_ctx, n_q_heads, n_kv_heads, head_dim, rank, meta_heads, group_size, top_k,
+               kv_dtype, meta_dtype, q_dtype, scope=KVSWAP_SCOPE_KV_HEAD, kv_strides=(0, 0, 0),
+               meta_strides=(0, 0, 0)) -> kvswap_shape:
+    return kvswap_shape(batch, n_ctx, n_q_heads, n_kv_heads, head_dim, rank, meta_heads, group_size, top_k,
+                        kv_dtype, meta_dtype, q_dtype, scope, *kv_strides, *meta_strides)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return getattr(stream, "cuda_stream", stream) or None
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise KVSwapError(status, where)
+
+
+def kvswap_workspace_bytes(shape: kvswap_shape) -> int:
+    return int(load().kvswap_workspace_bytes(ctypes.byref(shape)))
+
+
+def kvswap_validate_shape(shape: kvswap_shape) -> int:
+    return int(load().kvswap_validate_shape(ctypes.byref(shape)))
+
+
+def kvswap_project_keys(shape, K, proj, meta_out, n_begin, n_end, ws, stream=None) -> None:
+    _check(load().kvswap_project_keys(ctypes.byref(shape), _ptr(K), _ptr(proj), _ptr(meta_out), int(n_begin),
+                                      int(n_end), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                      _stream(stream)), "kvswap_project_keys")
+
+
+def kvswap_score_select(shape, q, proj, meta, group_idx, n_selected, group_scores_opt, ws, stream=None) -> None:
+    _check(load().kvswap_score_select(ctypes.byref(shape), _ptr(q), _ptr(proj), _ptr(meta), _ptr(group_idx),
+                                      _ptr(n_selected), _ptr(group_scores_opt), _ptr(ws),
+                                      0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "kvswap_score_select")
+
+
+def kvswap_sparse_decode(shape, q, K, V, group_idx, n_selected, out, lse_opt, ws, stream=None) -> None:
+    _check(load().kvswap_sparse_decode(ctypes.byref(shape), _ptr(q), _ptr(K), _ptr(V), _ptr(group_idx),
+                                       _ptr(n_selected), _ptr(out), _ptr(lse_opt), _ptr(ws),
+                                       0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
+           "kvswap_sparse_decode")
+
+
+def kvswap_version() -> int:
+    return int(load().kvswap_version())

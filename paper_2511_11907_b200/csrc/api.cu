@@ -1,0 +1,180 @@
+// C-ABI entry points of the kvswap library: host-side validation, workspace partition and
+// kernel sequencing.  No entry point allocates, synchronises or keeps state.
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace kvswap {
+
+static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+static int dtype_bytes(int t) {
+  switch (t) {
+    case KVSWAP_F32: return 4;
+    case KVSWAP_BF16: case KVSWAP_F16: return 2;
+    default: return 0;
+  }
+}
+
+int resolve(const kvswap_shape* s, Problem* p) {
+  if (s == nullptr) return KVSWAP_ERR_NULL;
+  if (s->batch < 1 || s->n_ctx < 1 || s->n_q_heads < 1 || s->n_kv_heads < 1 || s->group_size < 1 ||
+      s->top_k < 1 || s->rank < 1)
+    return KVSWAP_ERR_SHAPE;
+  if (s->n_q_heads % s->n_kv_heads != 0) return KVSWAP_ERR_SHAPE;
+  if (s->meta_heads != 1 && s->meta_heads != s->n_kv_heads) return KVSWAP_ERR_SHAPE;
+  if (s->scope != KVSWAP_SCOPE_KV_HEAD && s->scope != KVSWAP_SCOPE_ALL_HEADS) return KVSWAP_ERR_SHAPE;
+  if (s->n_ctx > (1 << 30) || s->batch > 65535 || s->n_q_heads > 4096) return KVSWAP_ERR_SHAPE;
+  const int ekv = dtype_bytes(s->kv_dtype), em = dtype_bytes(s->meta_dtype), eq = dtype_bytes(s->q_dtype);
+  if (ekv == 0 || em == 0 || eq == 0) return KVSWAP_ERR_DTYPE;
+  if (s->meta_dtype == KVSWAP_BF16) return KVSWAP_ERR_DTYPE;   // metadata is fp16 or fp32
+  if (s->q_dtype != KVSWAP_F32 && s->q_dtype != s->kv_dtype) return KVSWAP_ERR_DTYPE;  // q: fp32 or K/V's type
+  if (s->head_dim != 64 && s->head_dim != 128) return KVSWAP_ERR_UNSUPPORTED;
+  if (s->rank % 4 != 0 || s->rank > 256 || s->group_size > 1024) return KVSWAP_ERR_UNSUPPORTED;
+  if ((int64_t(s->rank) * em) % 16 != 0) return KVSWAP_ERR_ALIGN;
+  if ((int64_t(s->head_dim) * eq) % 16 != 0) return KVSWAP_ERR_ALIGN;
+
+  p->B = s->batch; p->N = s->n_ctx; p->Hq = s->n_q_heads; p->Hkv = s->n_kv_heads; p->d = s->head_dim;
+  p->r = s->rank; p->Hm = s->meta_heads; p->G = s->group_size; p->M = s->top_k;
+  p->kv_dtype = s->kv_dtype; p->meta_dtype = s->meta_dtype; p->q_dtype = s->q_dtype; p->scope = s->scope;
+
+  p->kv_sn = s->kv_stride_n ? s->kv_stride_n : p->d;
+  p->kv_sh = s->kv_stride_h ? s->kv_stride_h : int64_t(p->N) * p->kv_sn;
+  p->kv_sb = s->kv_stride_b ? s->kv_stride_b : int64_t(p->Hkv) * p->kv_sh;
+  p->meta_sn = s->meta_stride_n ? s->meta_stride_n : p->r;
+  p->meta_sh = s->meta_stride_h ? s->meta_stride_h : int64_t(p->N) * p->meta_sn;
+  p->meta_sb = s->meta_stride_b ? s->meta_stride_b : int64_t(p->Hm) * p->meta_sh;
+  if (p->kv_sn < p->d || p->kv_sh < 0 || p->kv_sb < 0 || p->meta_sn < p->r || p->meta_sh < 0 || p->meta_sb < 0)
+    return KVSWAP_ERR_SHAPE;
+  if ((p->kv_sn * ekv) % 16 || (p->kv_sh * ekv) % 16 || (p->kv_sb * ekv) % 16) return KVSWAP_ERR_ALIGN;
+  if ((p->meta_sn * em) % 16 || (p->meta_sh * em) % 16 || (p->meta_sb * em) % 16) return KVSWAP_ERR_ALIGN;
+
+  p->rho = p->Hq / p->Hkv;
+  p->S = (p->scope == KVSWAP_SCOPE_KV_HEAD) ? p->Hkv : 1;
+  p->NG = p->N / p->G;
+  p->Mp = std::min(p->M, p->NG);
+  p->Su = (p->Hm == 1) ? p->S : p->Hkv;
+  return KVSWAP_OK;
+}
+
+void plan_workspace(const Problem& p, Workspace* w) {
+  // sparse_decode: rho query heads share each K/V row; a CTA serves up to 4 of them per pass.
+  int rh = 1;
+  for (int c = 4; c >= 1; --c) if (p.rho % c == 0) { rh = c; break; }
+  w->heads_per_cta = rh;
+  const int64_t base = int64_t(p.B) * p.Hkv * (p.rho / rh);
+  const int64_t tokens = int64_t(p.Mp) * p.G + (p.N - int64_t(p.NG) * p.G);
+  int64_t splits = (int64_t(kNumSMs) * 4 + base - 1) / base;
+  splits = std::min<int64_t>(splits, (tokens + 63) / 64);
+  splits = std::max<int64_t>(1, std::min<int64_t>(splits, 256));
+  w->splits = int(splits);
+
+  size_t off = 256;  // first 256 bytes reserved
+  w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
+  w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * std::max(p.NG, 1));
+  w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
+  w->total = off;
+}
+
+static bool misaligned(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0; }
+
+}  // namespace kvswap
+
+using namespace kvswap;
+
+extern "C" {
+
+size_t kvswap_workspace_bytes(const kvswap_shape* shape) {
+  Problem p;
+  if (resolve(shape, &p) != KVSWAP_OK) return 0;
+  Workspace w;
+  plan_workspace(p, &w);
+  return w.total;
+}
+
+int kvswap_validate_shape(const kvswap_shape* shape) {
+  Problem p;
+  return resolve(shape, &p);
+}
+
+int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* proj, void* meta_out,
+                        int32_t n_begin, int32_t n_end, void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  Problem p;
+  int st = resolve(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  if (K == nullptr || proj == nullptr || meta_out == nullptr) return KVSWAP_ERR_NULL;
+  if (misaligned(K) || misaligned(proj) || misaligned(meta_out)) return KVSWAP_ERR_ALIGN;
+  if (n_begin < 0 || n_end < n_begin || n_end > p.N) return KVSWAP_ERR_SHAPE;
+  if (n_begin == n_end) return KVSWAP_OK;
+  cudaError_t e = launch_project_keys(p, K, proj, meta_out, n_begin, n_end, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+}
+
+int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
+                        int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
+                        size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  int st = resolve(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  if (q == nullptr || proj == nullptr || meta == nullptr || group_idx == nullptr || n_selected == nullptr ||
+      ws == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (misaligned(q) || misaligned(proj) || misaligned(meta) || misaligned(ws) ||
+      (reinterpret_cast<uintptr_t>(group_idx) & 3u) || (reinterpret_cast<uintptr_t>(n_selected) & 3u) ||
+      (group_scores_opt && misaligned(group_scores_opt)))
+    return KVSWAP_ERR_ALIGN;
+  Workspace w;
+  plan_workspace(p, &w);
+  if (ws_bytes < w.total) return KVSWAP_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(ws);
+  float* uq = reinterpret_cast<float*>(base + w.off_uq);
+  float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
+
+  cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
+  if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, stream);
+  if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
+  return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+}
+
+int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K, const void* V,
+                         const int32_t* group_idx, const int32_t* n_selected, float* out, float* lse_opt,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  int st = resolve(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  if (q == nullptr || K == nullptr || V == nullptr || group_idx == nullptr || n_selected == nullptr ||
+      out == nullptr || ws == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (misaligned(q) || misaligned(K) || misaligned(V) || misaligned(out) || misaligned(ws) ||
+      (reinterpret_cast<uintptr_t>(group_idx) & 3u) || (reinterpret_cast<uintptr_t>(n_selected) & 3u) ||
+      (lse_opt && (reinterpret_cast<uintptr_t>(lse_opt) & 3u)))
+    return KVSWAP_ERR_ALIGN;
+  Workspace w;
+  plan_workspace(p, &w);
+  if (ws_bytes < w.total) return KVSWAP_ERR_WORKSPACE;
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_partial);
+  cudaError_t e = launch_sparse_decode(p, w, q, K, V, group_idx, n_selected, partial, out, lse_opt,
+                                       static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+}
+
+const char* kvswap_status_string(int status) {
+  switch (status) {
+    case KVSWAP_OK: return "ok";
+    case KVSWAP_ERR_NULL: return "a required pointer is NULL";
+    case KVSWAP_ERR_SHAPE: return "invalid shape, stride, range or enum value";
+    case KVSWAP_ERR_DTYPE: return "unknown or unsupported dtype";
+    case KVSWAP_ERR_ALIGN: return "pointer or row size is not 16-byte aligned";
+    case KVSWAP_ERR_WORKSPACE: return "workspace smaller than kvswap_workspace_bytes()";
+    case KVSWAP_ERR_UNSUPPORTED: return "shape outside the implemented range";
+    case KVSWAP_ERR_CUDA: return "CUDA runtime or launch error";
+    case KVSWAP_ERR_INDEX: return "group index out of range";
+    default: return "unknown status";
+  }
+}
+
+int kvswap_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,90 @@
+// Shared declarations of the kvswap CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvswap.h"
+
+namespace kvswap {
+
+constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs; grids are sized in multiples of this.
+
+// Shape with every "0 = dense" stride resolved and the derived sizes filled in.
+struct Problem {
+  int B, N, Hq, Hkv, d, r, Hm, G, M;
+  int kv_dtype, meta_dtype, q_dtype, scope;
+  int64_t kv_sb, kv_sh, kv_sn;
+  int64_t meta_sb, meta_sh, meta_sn;
+  int rho;   // H_q / H_kv
+  int S;     // selections per sequence
+  int NG;    // complete groups
+  int Mp;    // min(M, NG)
+  int Su;    // rows of the low-rank query buffer per sequence (see score_pool.cu)
+};
+
+// Partition of the caller's workspace (byte offsets, each 256-byte aligned).
+struct Workspace {
+  size_t off_uq;       // float [B, Su, r]       summed low-rank queries
+  size_t off_scores;   // float [B, S, NG]       group scores R (when the caller passes no buffer)
+  size_t off_partial;  // float [B, Hq, splits, d + 2]  split-K partials (m, l, acc[d])
+  size_t total;
+  int splits;          // split-K factor of sparse_decode for this shape
+  int heads_per_cta;   // query heads sharing one K/V pass in sparse_decode
+};
+
+int resolve(const kvswap_shape* s, Problem* p);            // validation; returns kvswap_status
+void plan_workspace(const Problem& p, Workspace* w);
+
+// Kernel launchers (each returns a cudaError_t from the launch).
+cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta,
+                                int n_begin, int n_end, cudaStream_t st);
+cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* proj, float* uq,
+                                 cudaStream_t st);
+cudaError_t launch_score_pool(const Problem& p, const float* uq, const void* meta, float* scores,
+                              cudaStream_t st);
+cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* group_idx,
+                               int32_t* n_selected, cudaStream_t st);
+cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K,
+                                 const void* V, const int32_t* group_idx, const int32_t* n_selected,
+                                 float* partial, float* out, float* lse, cudaStream_t st);
+
+// ------------------------------------------------------------------------------------------
+// Device helpers: 16-byte vector loads of storage types, widened to fp32.
+// ------------------------------------------------------------------------------------------
+template <typename T> struct Elt;
+template <> struct Elt<float> { static constexpr int kPer16B = 4; };
+template <> struct Elt<__nv_bfloat16> { static constexpr int kPer16B = 8; };
+template <> struct Elt<__half> { static constexpr int kPer16B = 8; };
+
+__device__ __forceinline__ void widen16B(const uint4& v, float (&f)[4], float) {
+  f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+  f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void widen16B(const uint4& v, float (&f)[8], __nv_bfloat16) {
+  // bf16 -> fp32 is a 16-bit shift of the bit pattern.
+  f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+  f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+  f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+  f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+__device__ __forceinline__ void widen16B(const uint4& v, float (&f)[8], __half) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x; f[2 * i + 1] = t.y;
+  }
+}
+
+// 16-byte read-only global load that does not allocate in L1 (streamed once).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+}  // namespace kvswap

@@ -171,7 +171,7 @@ def adapter_from_calibration(calib: np.ndarray, n_kv_heads: int, head_dim: int, 
         flat = c64.reshape(rows, n_kv_heads * head_dim)
         _, _, vt = np.linalg.svd(flat, full_matrices=False)
         a = _fix_signs(vt[:rank].T)                       # [(H_kv*d), r]
-        return a.reshape(n_kv_heads, head_dim, rank).astype(dtype)
+        return np.ascontiguousarray(a.reshape(n_kv_heads, head_dim, rank), dtype=dtype)
     out = np.empty((n_kv_heads, head_dim, rank), dtype=dtype)
     for g in range(n_kv_heads):
         _, _, vt = np.linalg.svd(c64[:, g, :], full_matrices=False)

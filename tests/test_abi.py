@@ -1,0 +1,95 @@
+"""The C-ABI library loads, exports every symbol declared in include/kvswap.h, and its host-side
+validation returns the documented status codes.  No GPU needed: no compute entry point is reached
+with valid arguments."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2511_11907_b200 import binding as kv
+from paper_2511_11907_b200 import build as kvbuild
+from paper_2511_11907_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    kvbuild.build()
+    return kv.load()
+
+
+def _declared_functions():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(kvswap_\w+)\s*\(", text))
+    return names
+
+
+def good_shape(**kw):
+    args = dict(batch=2, n_ctx=1024, n_q_heads=8, n_kv_heads=2, head_dim=64, rank=16, meta_heads=1,
+                group_size=4, top_k=32, kv_dtype=W.F32, meta_dtype=W.F32, q_dtype=W.F32)
+    args.update(kw)
+    return kv.make_shape(**args)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    declared = _declared_functions()
+    assert {"kvswap_project_keys", "kvswap_score_select", "kvswap_sparse_decode",
+            "kvswap_workspace_bytes", "kvswap_status_string"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in include/ but not exported"
+
+
+def test_struct_layout_matches_header():
+    assert ctypes.sizeof(kv.kvswap_shape) == 13 * 4 + 4 + 6 * 8   # 13 int32, padding, 6 int64
+
+
+def test_validation_status_codes(lib):
+    assert kv.kvswap_validate_shape(good_shape()) == 0
+    assert kv.kvswap_workspace_bytes(good_shape()) > 0
+    bad = {
+        2: [dict(batch=0), dict(n_ctx=0), dict(n_q_heads=7), dict(meta_heads=3), dict(group_size=0),
+            dict(top_k=0), dict(scope=5), dict(kv_strides=(0, 0, 32))],
+        3: [dict(kv_dtype=9), dict(meta_dtype=W.BF16), dict(kv_dtype=W.F32, q_dtype=W.BF16)],
+        4: [dict(rank=4, meta_dtype=W.F16), dict(kv_strides=(0, 0, 66))],
+        6: [dict(head_dim=96), dict(rank=18), dict(rank=512), dict(group_size=2048)],
+    }
+    for code, cases in bad.items():
+        for c in cases:
+            s = good_shape(**c)
+            assert kv.kvswap_validate_shape(s) == code, (code, c)
+            assert kv.kvswap_workspace_bytes(s) == 0
+    assert lib.kvswap_validate_shape(None) == 1
+
+
+def test_entry_points_reject_null_and_small_workspace_without_touching_the_gpu(lib):
+    s = good_shape()
+    ref = ctypes.byref(s)
+    assert lib.kvswap_project_keys(ref, None, None, None, 0, 8, None, 0, None) == 1
+    assert lib.kvswap_score_select(ref, None, None, None, None, None, None, None, 0, None) == 1
+    assert lib.kvswap_sparse_decode(ref, None, None, None, None, None, None, None, None, 0, None) == 1
+    fake = ctypes.c_void_p(4096)                     # aligned, never dereferenced on these paths
+    assert lib.kvswap_project_keys(ref, fake, fake, fake, 8, 4, None, 0, None) == 2       # bad range
+    assert lib.kvswap_project_keys(ref, fake, fake, fake, 0, 4096, None, 0, None) == 2    # beyond N
+    assert lib.kvswap_project_keys(ref, fake, fake, fake, 5, 5, None, 0, None) == 0       # empty: no-op
+    assert lib.kvswap_project_keys(ref, ctypes.c_void_p(4100), fake, fake, 0, 8, None, 0, None) == 4
+    assert lib.kvswap_score_select(ref, fake, fake, fake, fake, fake, None, fake, 16, None) == 5
+    assert lib.kvswap_sparse_decode(ref, fake, fake, fake, fake, fake, fake, None, fake, 16, None) == 5
+
+
+def test_status_strings_and_version(lib):
+    seen = {kv.status_string(i) for i in range(9)}
+    assert len(seen) == 9 and "ok" in seen
+    assert kv.status_string(123) == "unknown status"
+    assert kv.kvswap_version() >= 100
+
+
+def test_workspace_grows_with_the_problem(lib):
+    small = kv.kvswap_workspace_bytes(good_shape())
+    big = kv.kvswap_workspace_bytes(good_shape(batch=8, n_ctx=65536))
+    assert big > small

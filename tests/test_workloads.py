@@ -59,3 +59,9 @@ def test_random_walk_queries_are_correlated():
     a, b = li.q_walk[0].ravel().astype(np.float64), li.q_walk[1].ravel().astype(np.float64)
     assert abs(np.corrcoef(a, b)[0, 1] - 0.95) < 0.02
     assert np.array_equal(li.q_walk[0], li.q)
+
+
+def test_generated_arrays_are_c_contiguous():
+    li = W.make_layer(W.CONFIGS[1], 0, meta_heads=1)
+    for a in (li.K, li.V, li.q, li.K_raw, li.V_raw, li.q_raw, li.proj):
+        assert a.flags["C_CONTIGUOUS"]
