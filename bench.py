@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the KVSwap decode hot path (predictor + sparse decode attention) on B200.
+
+A *step* is one decode step over all L layers of the workload: per layer, kvswap_score_select
+(low-rank scoring -> head sum -> group max -> top-k) followed by kvswap_sparse_decode (gather +
+split-K online-softmax attention + combine), on one stream, through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--meta joint|per_head]
+    python bench.py --impl reference ...      # the CPU oracle timed on the host cores
+
+Prints ONE JSON line (rank 0).  `value` is decode steps/s with every input resident in HBM;
+`e2e` is the same step driven through kvswap_decode_step_host with the step's queries in pinned
+host memory and its outputs read back, both copies inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2511_11907_b200 import workloads as W  # noqa: E402
+
+METRIC = "decode_steps_per_sec"
+UNIT = "steps/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--meta", choices=["joint", "per_head"], default="joint")
+    ap.add_argument("--scope", choices=["kv_head", "all_heads"], default="kv_head")
+    ap.add_argument("--layers", type=int, default=None, help="override L (debugging only; reported)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def workload_name(wl, args):
+    n = {W.F32: "fp32", W.BF16: "bf16", W.F16: "fp16"}
+    return (f"config{wl.config}: L={wl.layers} B={wl.batch} N={wl.n_ctx} Hq/Hkv={wl.n_q_heads}/{wl.n_kv_heads} "
+            f"d={wl.head_dim} r={wl.rank} G={wl.group_size} M={wl.top_k} kv={n[wl.kv_dtype]} meta={n[wl.meta_dtype]} "
+            f"layout={args.meta} scope={args.scope}")
+
+
+# --------------------------------------------------------------------------------------------
+# Clock sampling during the timed region
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            import torch
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            ident = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            ident = str(device_index)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50", "-i", ident],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t_begin: float, t_end: float):
+        """Summary of the samples taken in [t_begin, t_end] (wall clock); if the region was too
+        short to catch any, of all samples taken while the GPU ran the same step loop."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        rows = []
+        for line in self.file:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                ts = time.mktime(time.strptime(parts[0].split(".")[0], "%Y/%m/%d %H:%M:%S")) + float("0." + parts[0].split(".")[1])
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:8]))
+            except Exception:
+                continue
+        self.file.close()
+        os.unlink(self.file.name)
+        inside = [r for r in rows if t_begin - 0.05 <= r[0] <= t_end + 0.05]
+        used, where = (inside, "timed region") if inside else (rows, "whole step loop (timed region shorter than one sample)")
+        if not used:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in used for n, v in zip(names, r[3]) if v == "Active"})
+        return {"sm_mhz": statistics.median(r[1] for r in used), "sm_max_mhz": max(r[2] for r in used),
+                "reasons": reasons, "samples": len(used), "window": where}
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and the --impl reference arm)
+# --------------------------------------------------------------------------------------------
+def oracle_unit_time(K, V, q, proj, meta, wl, scope_name, heads=None):
+    """Seconds the oracle needs for one (layer, sequence) unit: score_select then attend.
+    K, V [1,H_kv,N,d]; q [1,H_q,d]; meta [1,H_m,N,r].  `heads` limits the unit to the first
+    KV heads (per-head work is independent; the caller scales)."""
+    from oracle import kvswap_oracle as O
+    if heads is not None and heads < wl.n_kv_heads:
+        rho = wl.rho
+        K, V, q, proj = K[:, :heads], V[:, :heads], q[:, :heads * rho], proj[:heads]
+        if meta.shape[1] != 1:
+            meta = meta[:, :heads]
+    t0 = time.perf_counter()
+    idx, _ = O.score_select(q, proj, meta, wl.group_size, wl.top_k, scope_name)
+    O.attend(q, K, V, idx, wl.group_size, scope_name)
+    return time.perf_counter() - t0
+
+
+def host_unit_inputs(wl, layer, meta_heads, seed_salt=0):
+    """One sequence of one layer drawn on the host (numpy) + oracle metadata (not timed)."""
+    from oracle import kvswap_oracle as O
+    one = wl.reduced(wl.name + "-unit", batch=1, walk_steps=1)
+    li = W.make_layer(one, layer, meta_heads)
+    meta = O.project_keys(li.K, li.proj, meta_heads, "f16" if wl.meta_dtype == W.F16 else "f32")
+    return li.K, li.V, li.q, li.proj, meta
+
+
+def threads_used():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def run_reference(args, wl):
+    """The oracle as it stands, on the host cores, on a bounded sample of the same workload."""
+    steps = args.steps if args.steps is not None else 5
+    warmup = args.warmup if args.warmup is not None else 1
+    meta_heads = 1 if args.meta == "joint" else wl.n_kv_heads
+    scope_name = args.scope
+    K, V, q, proj, meta = host_unit_inputs(wl, 0, meta_heads)
+    # size the per-step sample so that the whole run stays within a few minutes
+    t_probe = oracle_unit_time(K, V, q, proj, meta, wl, scope_name, heads=1)
+    budget = 150.0 / max(1, steps + warmup)
+    heads = int(max(1, min(wl.n_kv_heads, budget // max(t_probe, 1e-3))))
+    if scope_name == "all_heads":
+        heads = wl.n_kv_heads
+    for _ in range(warmup):
+        oracle_unit_time(K, V, q, proj, meta, wl, scope_name, heads)
+    times = [oracle_unit_time(K, V, q, proj, meta, wl, scope_name, heads) for _ in range(steps)]
+    t_unit = statistics.mean(times) * (wl.n_kv_heads / heads)
+    ms_per_step = t_unit * wl.layers * wl.batch * 1e3
+    value = 1e3 / ms_per_step
+    sample = (f"each timed step = oracle score_select+attend on 1 of {wl.layers} layers x 1 of {wl.batch} sequences "
+              f"x {heads} of {wl.n_kv_heads} KV heads; scaled linearly to the full step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(wl, args)},
+        "keys_scored_per_sec": value * wl.batch * wl.n_ctx * wl.layers,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads_used(), "kind": "oracle", "sample": sample,
+                         "host_cores_available": len(os.sched_getaffinity(0))},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_11907_b200 import binding as kv
+    from paper_2511_11907_b200 import build as kvbuild
+    from paper_2511_11907_b200 import device_workload as DW
+    from paper_2511_11907_b200 import runtime as rt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py (impl=ours) needs a CUDA device: the kvswap hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if not os.path.exists(kv.LIB_PATH):
+        if rank == 0:
+            kvbuild.build()
+        if world > 1:
+            dist.barrier()
+    kv.load()
+
+    steps = args.steps if args.steps is not None else 400
+    warmup = max(3, args.warmup if args.warmup is not None else 20)
+    meta_heads = 1 if args.meta == "joint" else wl.n_kv_heads
+    scope = W.SCOPE_KV_HEAD if args.scope == "kv_head" else W.SCOPE_ALL_HEADS
+
+    dw = DW.build(wl, meta_heads, scope, device=dev, rank_offset=rank)
+    shape, L = dw.shape, wl.layers
+    ws = rt.alloc_workspace(shape, dev)
+    stream = torch.cuda.current_stream()
+
+    # ---- prefill: metadata build, timed separately (not part of the decode step) ----------------
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for l in range(L):
+        kv.kvswap_project_keys(shape, dw.K[l], dw.proj[l], dw.meta[l], 0, wl.n_ctx, ws)
+    ev1.record()
+    torch.cuda.synchronize()
+    prefill_ms = ev0.elapsed_time(ev1)
+
+    layers = dw.layer_tables()
+    S, M = shape.n_scopes, wl.top_k
+    idx = torch.empty((L, wl.batch, S, M), dtype=torch.int32, device=dev)
+    nsel = torch.empty((L, wl.batch, S), dtype=torch.int32, device=dev)
+    out = torch.empty((L, wl.batch, wl.n_q_heads, wl.head_dim), dtype=torch.float32, device=dev)
+    n_walk = dw.q_walk.shape[0]
+
+    def step(i, probe=None):
+        kv.kvswap_decode_step(shape, layers, dw.q_walk[i % n_walk], out, None, idx, nsel, ws, probe)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    for i in range(warmup):
+        step(i)
+
+    # ---- timed region: K steps, inputs resident in HBM ----------------------------------------------
+    probes = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+               torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    probe_structs = [kv.make_probe(i % L, *probes[i]) for i in range(steps)]
+    prev_sel, overlaps = None, []
+    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    wall0 = time.time()
+    t_start.record()
+    for i in range(steps):
+        step(warmup + i, probe_structs[i])
+    t_stop.record()
+    sync_all()
+    wall1 = time.time()
+    elapsed_ms = t_start.elapsed_time(t_stop)
+    select_ms = [p[0].elapsed_time(p[1]) for p in probes]
+    decode_ms = [p[1].elapsed_time(p[2]) for p in probes]
+
+    # ---- selection overlap between consecutive steps (Sec. 4.4.2), outside the timed region ----
+    for i in range(min(8, n_walk)):
+        step(i)
+        torch.cuda.synchronize()
+        cur = idx[0].clone()
+        if prev_sel is not None:
+            a, b = cur.reshape(-1, M), prev_sel.reshape(-1, M)
+            hit = (a.unsqueeze(2) == b.unsqueeze(1)).any(dim=2) & (a >= 0)
+            overlaps.append(float(hit.float().sum() / (a >= 0).float().sum()))
+        prev_sel = cur
+
+    # ---- end to end: host queries in, host outputs back, every step ---------------------------------
+    q_host = torch.empty((n_walk,) + tuple(dw.q_walk.shape[1:]), dtype=dw.q_walk.dtype).pin_memory()
+    q_host.copy_(dw.q_walk)
+    out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    q_dev = torch.empty_like(dw.q_walk[0])
+    e2e_steps = steps
+
+    def step_host(i):
+        kv.kvswap_decode_step_host(shape, layers, q_host[i % n_walk], out_host, q_dev, out, idx, nsel, ws)
+        stream.synchronize()                     # the step's result is needed before the next token
+
+    for i in range(3):
+        step_host(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for i in range(e2e_steps):
+        step_host(i)
+    e1.record()
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(wall0, wall1) if sampler else None
+
+    # ---- max over ranks ----------------------------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    esz = {W.F32: 4, W.BF16: 2, W.F16: 2}
+    Mp = min(M, wl.n_groups)
+    ms_per_step = elapsed_ms / steps
+    value = world * 1e3 / ms_per_step
+    keys_per_step = wl.batch * wl.n_ctx * L
+    decode_bytes = 2 * wl.batch * wl.n_kv_heads * Mp * wl.group_size * wl.head_dim * esz[wl.kv_dtype] + wl.batch * S * M * 4
+    select_bytes = (wl.batch * meta_heads * wl.n_ctx * wl.rank * esz[wl.meta_dtype] + 2 * wl.batch * S * wl.n_groups * 4
+                    + wl.batch * S * M * 4)
+    peak, peak_kind = measured_peak()
+    dec_ms, sel_ms = statistics.mean(decode_ms), statistics.mean(select_ms)
+    dec_gbs, sel_gbs = decode_bytes / dec_ms / 1e6, select_bytes / sel_ms / 1e6
+    q_bytes = q_host[0].numel() * q_host.element_size()
+    out_bytes = out_host.numel() * 4
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(wl, args), "parallelism": f"batch shards x{world}, no collective",
+                   "global_batch": wl.batch * world, "layers_resident": dw.layers_resident,
+                   "l2": "inputs larger than L2: every step streams all layers' metadata and gathers from "
+                         f"{dw.layers_resident} distinct KV stores (>> 126 MB) before any buffer repeats",
+                   "kv_resident_gb": round(dw.layers_resident * 2 * dw.K[0].numel() * esz[wl.kv_dtype] / 1e9, 1)},
+        "keys_scored_per_sec": value * keys_per_step,
+        "e2e": {"value": world * 1e3 * e2e_steps / e2e_ms, "unit": UNIT, "h2d_bytes_per_step": q_bytes,
+                "d2h_bytes_per_step": out_bytes, "steps": e2e_steps},
+        "gpu_launches": 5 * L * steps,
+        "roofline": {"bound": "hbm", "kernel": "kvswap_sparse_decode (gather split-K + combine)",
+                     "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": None, "algorithmic_bytes_per_launch": decode_bytes, "avg_ms": dec_ms,
+                     "frac_of_nominal_8000": dec_gbs / 8000.0},
+        "roofline_score_select": {"bound": "hbm", "kernel": "kvswap_score_select (lowrank_query + score_pool + topk)",
+                                  "achieved": sel_gbs, "peak": peak, "unit": "GB/s", "frac": sel_gbs / peak,
+                                  "algorithmic_bytes_per_launch": select_bytes, "avg_ms": sel_ms},
+        "prefill": {"project_keys_ms_all_layers": prefill_ms,
+                    "keys_projected_per_sec": keys_per_step / prefill_ms * 1e3,
+                    "read_gbs": L * wl.batch * wl.n_kv_heads * wl.n_ctx * wl.head_dim * esz[wl.kv_dtype] / prefill_ms / 1e6},
+        "selection_overlap_ratio": statistics.mean(overlaps) if overlaps else None,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(wl, dw, meta_heads, args.scope, rt)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wl, dw, meta_heads, scope_name, rt):
+    """The oracle on (layer, sequence) units of the resident workload until ~10 s are spent."""
+    units, spent, t_units = 0, 0.0, []
+    while spent < 10.0 and units < wl.layers * wl.batch:
+        l, b = units % wl.layers, (units // wl.layers) % wl.batch
+        K = rt.to_host_f32(dw.K[l][b:b + 1])
+        V = rt.to_host_f32(dw.V[l][b:b + 1])
+        q = rt.to_host_f32(dw.q_walk[0, l, b:b + 1])
+        meta = rt.to_host_f32(dw.meta[l][b:b + 1])
+        proj = dw.proj[l].cpu().numpy()
+        t = oracle_unit_time(K, V, q, proj, meta, wl, scope_name)
+        t_units.append(t)
+        spent += t
+        units += 1
+    t_step = statistics.mean(t_units) * wl.layers * wl.batch
+    return {"value": 1.0 / t_step, "unit": UNIT, "cores": threads_used(), "kind": "oracle",
+            "sample": f"{units} (layer, sequence) units of the same workload ({spent:.1f} s of oracle time), "
+                      f"scaled to L*B = {wl.layers * wl.batch} units per step",
+            "host_cores_available": len(os.sched_getaffinity(0))}
+
+
+def main():
+    args = parse_args()
+    wl = W.CONFIGS[args.config]
+    if args.layers is not None:
+        wl = wl.reduced(wl.name + f"-L{args.layers}", layers=args.layers)
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, wl)
+        return
+    run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -133,6 +133,58 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
                          const int32_t* group_idx, const int32_t* n_selected,
                          float* out, float* lse_opt, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/*
+ * Per-layer tensors of a model with L layers that all share one kvswap_shape.  Each member is a
+ * HOST array of L DEVICE pointers: K[l], V[l] are [B, H_kv, N, d]; meta[l] is [B, H_m, N, r];
+ * proj[l] is [H_kv, d, r] fp32.
+ */
+typedef struct {
+  int32_t n_layers;
+  const void* const* K;
+  const void* const* V;
+  const void* const* meta;
+  const float* const* proj;
+} kvswap_layers;
+
+/*
+ * Optional timing probe of kvswap_decode_step: for layer `layer`, CUDA events (cudaEvent_t passed
+ * as void*, created with timing enabled by the caller) are recorded on the stream before
+ * score_select (ev_begin), between score_select and sparse_decode (ev_mid) and after
+ * sparse_decode (ev_end).  NULL events are skipped.
+ */
+typedef struct {
+  int32_t layer;
+  void* ev_begin;
+  void* ev_mid;
+  void* ev_end;
+} kvswap_probe;
+
+/*
+ * One decode step of the predictor + sparse attention (Sec. 4.4, decoding): for l = 0..L-1, in
+ * order on `cuda_stream`, kvswap_score_select then kvswap_sparse_decode on layer l, with
+ *   q          [L, B, H_q, d] q_dtype  (the same query scores and attends; device)
+ *   out        [L, B, H_q, d] fp32     (device)
+ *   lse_opt    NULL or [L, B, H_q] fp32
+ *   group_idx  [L, B, S, M] int32, n_selected [L, B, S] int32: the selections of this step, kept
+ *              per layer so that the caller can compare consecutive steps (Sec. 4.4.2).
+ * `ws` is shared by all layers (size: kvswap_workspace_bytes).  probe_opt may be NULL.
+ */
+int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q,
+                       float* out, float* lse_opt, int32_t* group_idx, int32_t* n_selected,
+                       void* ws, size_t ws_bytes, const kvswap_probe* probe_opt, void* cuda_stream);
+
+/*
+ * The same step for callers whose queries and outputs live in HOST memory: q_host
+ * [L, B, H_q, d] q_dtype is copied to the device buffer q_dev, the step runs, and out_dev is
+ * copied to out_host [L, B, H_q, d] fp32, all asynchronously on `cuda_stream` (use pinned host
+ * memory for the copies to overlap; the call returns before they complete).  q_dev, out_dev,
+ * group_idx, n_selected and ws are caller-provided device buffers as in kvswap_decode_step.
+ */
+int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* layers,
+                            const void* q_host, float* out_host, void* q_dev, float* out_dev,
+                            int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
+                            void* cuda_stream);
+
 /* Static, NUL-terminated description of a kvswap_status value. */
 const char* kvswap_status_string(int status);
 

@@ -128,3 +128,74 @@ def kvswap_sparse_decode(shape, q, K, V, group_idx, n_selected, out, lse_opt, ws
 
 def kvswap_version() -> int:
     return int(load().kvswap_version())
+
+
+# ------------------------------------------------------------------------------------------------
+# Whole decode step over L layers
+# ------------------------------------------------------------------------------------------------
+class kvswap_layers(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("K", ctypes.POINTER(ctypes.c_void_p)),
+                ("V", ctypes.POINTER(ctypes.c_void_p)), ("meta", ctypes.POINTER(ctypes.c_void_p)),
+                ("proj", ctypes.POINTER(ctypes.c_void_p))]
+
+
+class kvswap_probe(ctypes.Structure):
+    _fields_ = [("layer", ctypes.c_int32), ("ev_begin", ctypes.c_void_p), ("ev_mid", ctypes.c_void_p),
+                ("ev_end", ctypes.c_void_p)]
+
+
+def make_layers(K, V, meta, proj) -> kvswap_layers:
+    """Pointer tables for lists of per-layer device tensors.  The returned struct keeps the
+    tensors and the tables alive."""
+    n = len(K)
+    assert len(V) == n and len(meta) == n and len(proj) == n
+
+    def table(ts):
+        return (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+
+    tabs = [table(K), table(V), table(meta), table(proj)]
+    layers = kvswap_layers(n, *[ctypes.cast(t, ctypes.POINTER(ctypes.c_void_p)) for t in tabs])
+    layers._keep = (tabs, list(K), list(V), list(meta), list(proj))
+    return layers
+
+
+def make_probe(layer: int, ev_begin=None, ev_mid=None, ev_end=None) -> kvswap_probe:
+    """Probe from torch.cuda.Event objects created with enable_timing=True.  An event's handle
+    exists only once it has been recorded, so fresh events are recorded once here."""
+    def handle(ev):
+        if ev is None:
+            return None
+        if not ev.cuda_event:
+            ev.record()
+        return ev.cuda_event
+    return kvswap_probe(int(layer), handle(ev_begin), handle(ev_mid), handle(ev_end))
+
+
+def _declare_step(lib):
+    if getattr(lib, "_step_declared", False):
+        return lib
+    V, SZ = ctypes.c_void_p, ctypes.c_size_t
+    P, PL, PP = ctypes.POINTER(kvswap_shape), ctypes.POINTER(kvswap_layers), ctypes.POINTER(kvswap_probe)
+    lib.kvswap_decode_step.restype = ctypes.c_int
+    lib.kvswap_decode_step.argtypes = [P, PL, V, V, V, V, V, V, SZ, PP, V]
+    lib.kvswap_decode_step_host.restype = ctypes.c_int
+    lib.kvswap_decode_step_host.argtypes = [P, PL, V, V, V, V, V, V, V, SZ, V]
+    lib._step_declared = True
+    return lib
+
+
+def kvswap_decode_step(shape, layers, q, out, lse_opt, group_idx, n_selected, ws, probe_opt=None, stream=None) -> None:
+    lib = _declare_step(load())
+    _check(lib.kvswap_decode_step(ctypes.byref(shape), ctypes.byref(layers), _ptr(q), _ptr(out), _ptr(lse_opt),
+                                  _ptr(group_idx), _ptr(n_selected), _ptr(ws), ws.numel() * ws.element_size(),
+                                  None if probe_opt is None else ctypes.byref(probe_opt), _stream(stream)),
+           "kvswap_decode_step")
+
+
+def kvswap_decode_step_host(shape, layers, q_host, out_host, q_dev, out_dev, group_idx, n_selected, ws,
+                            stream=None) -> None:
+    """q_host / out_host are CPU tensors (pinned for asynchronous copies)."""
+    lib = _declare_step(load())
+    _check(lib.kvswap_decode_step_host(ctypes.byref(shape), ctypes.byref(layers), _ptr(q_host), _ptr(out_host),
+                                       _ptr(q_dev), _ptr(out_dev), _ptr(group_idx), _ptr(n_selected), _ptr(ws),
+                                       ws.numel() * ws.element_size(), _stream(stream)), "kvswap_decode_step_host")

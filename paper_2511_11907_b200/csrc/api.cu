@@ -160,6 +160,67 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 
+static int check_layers(const kvswap_layers* layers) {
+  if (layers == nullptr || layers->K == nullptr || layers->V == nullptr || layers->meta == nullptr ||
+      layers->proj == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (layers->n_layers < 1) return KVSWAP_ERR_SHAPE;
+  return KVSWAP_OK;
+}
+
+int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q, float* out,
+                       float* lse_opt, int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
+                       const kvswap_probe* probe_opt, void* cuda_stream) {
+  Problem p;
+  int st = resolve(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  st = check_layers(layers);
+  if (st != KVSWAP_OK) return st;
+  if (q == nullptr || out == nullptr || group_idx == nullptr || n_selected == nullptr) return KVSWAP_ERR_NULL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t q_bytes = size_t(p.B) * p.Hq * p.d * dtype_bytes(p.q_dtype);
+  const size_t out_elems = size_t(p.B) * p.Hq * p.d;
+  const size_t idx_elems = size_t(p.B) * p.S * p.M, nsel_elems = size_t(p.B) * p.S;
+  for (int l = 0; l < layers->n_layers; ++l) {
+    const bool probed = probe_opt != nullptr && probe_opt->layer == l;
+    const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+    int32_t* idx_l = group_idx + size_t(l) * idx_elems;
+    int32_t* nsel_l = n_selected + size_t(l) * nsel_elems;
+    if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), stream);
+    st = kvswap_score_select(shape, ql, layers->proj[l], layers->meta[l], idx_l, nsel_l, nullptr, ws, ws_bytes,
+                             cuda_stream);
+    if (st != KVSWAP_OK) return st;
+    if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), stream);
+    st = kvswap_sparse_decode(shape, ql, layers->K[l], layers->V[l], idx_l, nsel_l, out + size_t(l) * out_elems,
+                              lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes, cuda_stream);
+    if (st != KVSWAP_OK) return st;
+    if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
+  }
+  return KVSWAP_OK;
+}
+
+int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* layers, const void* q_host,
+                            float* out_host, void* q_dev, float* out_dev, int32_t* group_idx,
+                            int32_t* n_selected, void* ws, size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  int st = resolve(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  st = check_layers(layers);
+  if (st != KVSWAP_OK) return st;
+  if (q_host == nullptr || out_host == nullptr || q_dev == nullptr || out_dev == nullptr) return KVSWAP_ERR_NULL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t L = size_t(layers->n_layers);
+  const size_t q_bytes = L * p.B * p.Hq * p.d * dtype_bytes(p.q_dtype);
+  const size_t out_bytes = L * p.B * p.Hq * p.d * sizeof(float);
+  if (cudaMemcpyAsync(q_dev, q_host, q_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+  st = kvswap_decode_step(shape, layers, q_dev, out_dev, nullptr, group_idx, n_selected, ws, ws_bytes, nullptr,
+                          cuda_stream);
+  if (st != KVSWAP_OK) return st;
+  if (cudaMemcpyAsync(out_host, out_dev, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return KVSWAP_ERR_CUDA;
+  return KVSWAP_OK;
+}
+
 const char* kvswap_status_string(int status) {
   switch (status) {
     case KVSWAP_OK: return "ok";
