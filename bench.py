@@ -203,6 +203,7 @@ def run_ours(args, wl):
     from paper_2511_11907_b200 import build as kvbuild
     from paper_2511_11907_b200 import device_workload as DW
     from paper_2511_11907_b200 import runtime as rt
+    from paper_2511_11907_b200 import shard
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -225,7 +226,7 @@ def run_ours(args, wl):
     meta_heads = 1 if args.meta == "joint" else wl.n_kv_heads
     scope = W.SCOPE_KV_HEAD if args.scope == "kv_head" else W.SCOPE_ALL_HEADS
 
-    dw = DW.build(wl, meta_heads, scope, device=dev, rank_offset=rank)
+    dw = DW.build(wl, meta_heads, scope, device=dev, rank_offset=shard.rank_seed_offset(rank))
     shape, L = dw.shape, wl.layers
     ws = rt.alloc_workspace(shape, dev)
     stream = torch.cuda.current_stream()
@@ -313,10 +314,7 @@ def run_ours(args, wl):
     clocks = sampler.stop(wall0, wall1) if sampler else None
 
     # ---- max over ranks ----------------------------------------------------------------------------
-    if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    elapsed_ms, e2e_ms = shard.max_over_ranks([elapsed_ms, e2e_ms], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -325,7 +323,7 @@ def run_ours(args, wl):
     esz = {W.F32: 4, W.BF16: 2, W.F16: 2}
     Mp = min(M, wl.n_groups)
     ms_per_step = elapsed_ms / steps
-    value = world * 1e3 / ms_per_step
+    value = shard.aggregate_throughput(1.0, steps, elapsed_ms, world)
     keys_per_step = wl.batch * wl.n_ctx * L
     decode_bytes = 2 * wl.batch * wl.n_kv_heads * Mp * wl.group_size * wl.head_dim * esz[wl.kv_dtype] + wl.batch * S * M * 4
     select_bytes = (wl.batch * meta_heads * wl.n_ctx * wl.rank * esz[wl.meta_dtype] + 2 * wl.batch * S * wl.n_groups * 4
