@@ -55,7 +55,8 @@ typedef enum {
   KVSWAP_ERR_WORKSPACE = 5,   /* ws_bytes smaller than kvswap_workspace_bytes()              */
   KVSWAP_ERR_UNSUPPORTED = 6, /* valid request outside the implemented range                 */
   KVSWAP_ERR_CUDA = 7,        /* a CUDA runtime call or kernel launch failed                 */
-  KVSWAP_ERR_INDEX = 8        /* reserved: out-of-range group index seen by a checking build */
+  KVSWAP_ERR_INDEX = 8,       /* reserved: out-of-range group index seen by a checking build */
+  KVSWAP_ERR_STATIC_SCRATCH = 9 /* problem needs more than KVSWAP_STATIC_SCRATCH_BYTES of scratch */
 } kvswap_status;
 
 typedef enum { KVSWAP_F32 = 0, KVSWAP_BF16 = 1, KVSWAP_F16 = 2 } kvswap_dtype;
@@ -132,6 +133,36 @@ int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* p
 int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K, const void* V,
                          const int32_t* group_idx, const int32_t* n_selected,
                          float* out, float* lse_opt, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * kvswap_sparse_decode without a workspace argument.  (Library convenience: the paper has no
+ * counterpart; the computation is exactly that of kvswap_sparse_decode.)
+ *
+ * For callers that must not allocate device memory where they call the library and therefore
+ * have no scratch buffer to pass: e.g. a serving process whose memory manager took the whole GPU
+ * at start-up, or code running inside a host framework's enqueue callback where cudaMalloc is
+ * off limits because it synchronises the device and may fail late.  The split-K partials live
+ * in a buffer of KVSWAP_STATIC_SCRATCH_BYTES that is built into the library; every GPU that
+ * loads the library holds that much memory until the process exits.
+ *
+ *  - Inputs and outputs are the caller's, with the same meaning, layout and checks as in
+ *    kvswap_sparse_decode.  The call itself allocates and frees nothing.
+ *  - Problems whose partials, 4 * B * H_q * splits * (d + 2) bytes (splits as chosen by the
+ *    library for the shape, at most 256), exceed the buffer are refused with
+ *    KVSWAP_ERR_STATIC_SCRATCH before anything is launched.  All five benchmark configurations
+ *    fit (the largest needs about 2 MiB).
+ *  - The first call on each device looks up the buffer's device address (with that device
+ *    current) and caches it; make that first call outside of any stream capture.
+ *  - All calls on a device share the one buffer, and it keeps whatever the previous call left
+ *    there.  Nothing in it needs clearing (each call overwrites every slot it later reads), but
+ *    two calls that overlap on the GPU -- different streams, or threads -- race on it and give
+ *    wrong results: serialise them, or use kvswap_sparse_decode with separate workspaces.
+ */
+#define KVSWAP_STATIC_SCRATCH_BYTES (8u << 20)
+int kvswap_sparse_decode_static(const kvswap_shape* shape, const void* q, const void* K,
+                                const void* V, const int32_t* group_idx,
+                                const int32_t* n_selected, float* out, float* lse_opt,
+                                void* cuda_stream);
 
 /*
  * Per-layer tensors of a model with L layers that all share one kvswap_shape.  Each member is a

@@ -199,3 +199,22 @@ def kvswap_decode_step_host(shape, layers, q_host, out_host, q_dev, out_dev, gro
     _check(lib.kvswap_decode_step_host(ctypes.byref(shape), ctypes.byref(layers), _ptr(q_host), _ptr(out_host),
                                        _ptr(q_dev), _ptr(out_dev), _ptr(group_idx), _ptr(n_selected), _ptr(ws),
                                        ws.numel() * ws.element_size(), _stream(stream)), "kvswap_decode_step_host")
+
+
+KVSWAP_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def kvswap_sparse_decode_static(shape, q, K, V, group_idx, n_selected, out, lse_opt, stream=None) -> None:
+    """kvswap_sparse_decode for callers that cannot hand over a workspace (they are not allowed
+    to allocate device memory at the call site): the split-K partials go to a buffer built into
+    the library.  Problems too large for that buffer raise KVSwapError (status 9).  Calls on one
+    device share the buffer, so do not let two of them overlap on the GPU."""
+    lib = load()
+    if not getattr(lib, "_static_declared", False):
+        V_ = ctypes.c_void_p
+        lib.kvswap_sparse_decode_static.restype = ctypes.c_int
+        lib.kvswap_sparse_decode_static.argtypes = [ctypes.POINTER(kvswap_shape), V_, V_, V_, V_, V_, V_, V_, V_]
+        lib._static_declared = True
+    _check(lib.kvswap_sparse_decode_static(ctypes.byref(shape), _ptr(q), _ptr(K), _ptr(V), _ptr(group_idx),
+                                           _ptr(n_selected), _ptr(out), _ptr(lse_opt), _stream(stream)),
+           "kvswap_sparse_decode_static")

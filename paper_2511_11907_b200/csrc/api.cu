@@ -232,6 +232,7 @@ const char* kvswap_status_string(int status) {
     case KVSWAP_ERR_UNSUPPORTED: return "shape outside the implemented range";
     case KVSWAP_ERR_CUDA: return "CUDA runtime or launch error";
     case KVSWAP_ERR_INDEX: return "group index out of range";
+    case KVSWAP_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in static buffer holds";
     default: return "unknown status";
   }
 }
