@@ -56,7 +56,8 @@ typedef enum {
   KVSWAP_ERR_UNSUPPORTED = 6, /* valid request outside the implemented range                 */
   KVSWAP_ERR_CUDA = 7,        /* a CUDA runtime call or kernel launch failed                 */
   KVSWAP_ERR_INDEX = 8,       /* reserved: out-of-range group index seen by a checking build */
-  KVSWAP_ERR_STATIC_SCRATCH = 9 /* problem needs more than KVSWAP_STATIC_SCRATCH_BYTES of scratch */
+  KVSWAP_ERR_STATIC_SCRATCH = 9, /* problem needs more than KVSWAP_STATIC_SCRATCH_BYTES of scratch */
+  KVSWAP_ERR_TIMEOUT = 10     /* a kernel gave up a bounded wait; its outputs are invalid     */
 } kvswap_status;
 
 typedef enum { KVSWAP_F32 = 0, KVSWAP_BF16 = 1, KVSWAP_F16 = 2 } kvswap_dtype;
@@ -84,6 +85,20 @@ size_t kvswap_workspace_bytes(const kvswap_shape* shape);
 
 /* Validates `shape` exactly as the compute calls do (host only, touches no GPU). */
 int kvswap_validate_shape(const kvswap_shape* shape);
+
+/*
+ * Device status word.  The kernels stage K/V rows through shared memory with asynchronous copies
+ * and wait for them with a bounded number of attempts; a wait that runs out (which no valid
+ * input can cause) is recorded in the first word of the workspace instead of hanging the GPU.
+ *   kvswap_workspace_init     clears the word (asynchronously, on `cuda_stream`).  Call it once
+ *                             after allocating a workspace; a workspace that was never cleared
+ *                             computes correctly but reports garbage below.
+ *   kvswap_read_device_status waits for `cuda_stream` to drain (the only call of the library that
+ *                             synchronises), then returns KVSWAP_OK, or KVSWAP_ERR_TIMEOUT if a
+ *                             kernel using `ws` has given up a wait since the word was cleared.
+ */
+int kvswap_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);
+int kvswap_read_device_status(const void* ws, void* cuda_stream);
 
 /*
  * Metadata build, K_lr = Flatten(K) A (Sec. 4.2), for tokens n_begin <= n < n_end (prefill: the
@@ -147,8 +162,8 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
  *
  *  - Inputs and outputs are the caller's, with the same meaning, layout and checks as in
  *    kvswap_sparse_decode.  The call itself allocates and frees nothing.
- *  - Problems whose partials, 4 * B * H_q * splits * (d + 2) bytes (splits as chosen by the
- *    library for the shape, at most 256), exceed the buffer are refused with
+ *  - Problems whose partials, 256 + 4 * B * H_q * splits * (d + 2) bytes (splits as chosen by
+ *    the library for the shape, at most 256), exceed the buffer are refused with
  *    KVSWAP_ERR_STATIC_SCRATCH before anything is launched.  All five benchmark configurations
  *    fit (the largest needs about 2 MiB).
  *  - The first call on each device looks up the buffer's device address (with that device

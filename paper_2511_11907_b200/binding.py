@@ -67,6 +67,10 @@ def load() -> ctypes.CDLL:
     lib.kvswap_status_string.argtypes = [ctypes.c_int]
     lib.kvswap_version.restype = ctypes.c_int
     lib.kvswap_version.argtypes = []
+    lib.kvswap_workspace_init.restype = ctypes.c_int
+    lib.kvswap_workspace_init.argtypes = [V, SZ, V]
+    lib.kvswap_read_device_status.restype = ctypes.c_int
+    lib.kvswap_read_device_status.argtypes = [V, V]
     _lib = lib
     return lib
 
@@ -124,6 +128,16 @@ def kvswap_sparse_decode(shape, q, K, V, group_idx, n_selected, out, lse_opt, ws
                                        _ptr(n_selected), _ptr(out), _ptr(lse_opt), _ptr(ws),
                                        0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "kvswap_sparse_decode")
+
+
+def kvswap_workspace_init(ws, stream=None) -> None:
+    _check(load().kvswap_workspace_init(_ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "kvswap_workspace_init")
+
+
+def kvswap_read_device_status(ws, stream=None) -> int:
+    """Synchronises the stream; returns 0, or KVSWAP_ERR_TIMEOUT (10) if a kernel gave up a wait."""
+    return int(load().kvswap_read_device_status(_ptr(ws), _stream(stream)))
 
 
 def kvswap_version() -> int:

@@ -1,5 +1,6 @@
 // C-ABI entry points of the kvswap library: host-side validation, workspace partition and
-// kernel sequencing.  No entry point allocates, synchronises or keeps state.
+// kernel sequencing.  No entry point allocates or keeps state; only kvswap_read_device_status
+// synchronises.
 #include <algorithm>
 
 #include "common.cuh"
@@ -58,16 +59,7 @@ int resolve(const kvswap_shape* s, Problem* p) {
 }
 
 void plan_workspace(const Problem& p, Workspace* w) {
-  // sparse_decode: rho query heads share each K/V row; a CTA serves up to 4 of them per pass.
-  int rh = 1;
-  for (int c = 4; c >= 1; --c) if (p.rho % c == 0) { rh = c; break; }
-  w->heads_per_cta = rh;
-  const int64_t base = int64_t(p.B) * p.Hkv * (p.rho / rh);
-  const int64_t tokens = int64_t(p.Mp) * p.G + (p.N - int64_t(p.NG) * p.G);
-  int64_t splits = (int64_t(kNumSMs) * 4 + base - 1) / base;
-  splits = std::min<int64_t>(splits, (tokens + 63) / 64);
-  splits = std::max<int64_t>(1, std::min<int64_t>(splits, 256));
-  w->splits = int(splits);
+  plan_sparse_decode(p, w);
 
   size_t off = 256;  // first 256 bytes reserved
   w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
@@ -156,7 +148,7 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
   if (ws_bytes < w.total) return KVSWAP_ERR_WORKSPACE;
   float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_partial);
   cudaError_t e = launch_sparse_decode(p, w, q, K, V, group_idx, n_selected, partial, out, lse_opt,
-                                       static_cast<cudaStream_t>(cuda_stream));
+                                       static_cast<uint32_t*>(ws), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 
@@ -221,6 +213,22 @@ int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* laye
   return KVSWAP_OK;
 }
 
+int kvswap_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (ws == nullptr) return KVSWAP_ERR_NULL;
+  if (ws_bytes < 256) return KVSWAP_ERR_WORKSPACE;
+  return cudaMemsetAsync(ws, 0, 256, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? KVSWAP_OK
+                                                                                             : KVSWAP_ERR_CUDA;
+}
+
+int kvswap_read_device_status(const void* ws, void* cuda_stream) {
+  if (ws == nullptr) return KVSWAP_ERR_NULL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+  return word == 0 ? KVSWAP_OK : KVSWAP_ERR_TIMEOUT;
+}
+
 const char* kvswap_status_string(int status) {
   switch (status) {
     case KVSWAP_OK: return "ok";
@@ -233,6 +241,7 @@ const char* kvswap_status_string(int status) {
     case KVSWAP_ERR_CUDA: return "CUDA runtime or launch error";
     case KVSWAP_ERR_INDEX: return "group index out of range";
     case KVSWAP_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in static buffer holds";
+    case KVSWAP_ERR_TIMEOUT: return "a kernel gave up a bounded wait (device status word set)";
     default: return "unknown status";
   }
 }

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "kvswap.h"
 
 namespace kvswap {
@@ -33,10 +35,12 @@ struct Workspace {
   size_t total;
   int splits;          // split-K factor of sparse_decode for this shape
   int heads_per_cta;   // query heads sharing one K/V pass in sparse_decode
+  int depth;           // shared-memory stages per compute warp in sparse_decode
 };
 
 int resolve(const kvswap_shape* s, Problem* p);            // validation; returns kvswap_status
 void plan_workspace(const Problem& p, Workspace* w);
+void plan_sparse_decode(const Problem& p, Workspace* w);   // fills splits, heads_per_cta, depth
 
 // Kernel launchers (each returns a cudaError_t from the launch).
 cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta,
@@ -49,7 +53,25 @@ cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* g
                                int32_t* n_selected, cudaStream_t st);
 cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K,
                                  const void* V, const int32_t* group_idx, const int32_t* n_selected,
-                                 float* partial, float* out, float* lse, cudaStream_t st);
+                                 float* partial, float* out, float* lse, uint32_t* err, cudaStream_t st);
+
+// Launch with programmatic stream serialisation: the kernel may begin (up to its
+// griddepcontrol.wait) while the previous kernel in the stream is still draining.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // ------------------------------------------------------------------------------------------
 // Device helpers: 16-byte vector loads of storage types, widened to fp32.

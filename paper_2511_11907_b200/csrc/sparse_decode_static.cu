@@ -66,11 +66,13 @@ extern "C" int kvswap_sparse_decode_static(const kvswap_shape* shape, const void
     return KVSWAP_ERR_ALIGN;
   Workspace w;
   plan_workspace(p, &w);
-  const size_t need = sizeof(float) * size_t(p.B) * p.Hq * w.splits * (p.d + 2);
+  // The first 256 bytes hold the device status word, the partials follow.
+  const size_t need = 256 + sizeof(float) * size_t(p.B) * p.Hq * w.splits * (p.d + 2);
   if (need > size_t(KVSWAP_STATIC_SCRATCH_BYTES)) return KVSWAP_ERR_STATIC_SCRATCH;
   void* scratch = nullptr;
   if (scratch_address(&scratch) != cudaSuccess) return KVSWAP_ERR_CUDA;
-  cudaError_t e = launch_sparse_decode(p, w, q, K, V, group_idx, n_selected, static_cast<float*>(scratch), out,
-                                       lse_opt, static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = launch_sparse_decode(p, w, q, K, V, group_idx, n_selected,
+                                       reinterpret_cast<float*>(static_cast<char*>(scratch) + 256), out, lse_opt,
+                                       static_cast<uint32_t*>(scratch), static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }

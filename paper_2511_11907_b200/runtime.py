@@ -36,7 +36,9 @@ def alloc_workspace(shape: kv.kvswap_shape, device="cuda") -> torch.Tensor:
     n = kv.kvswap_workspace_bytes(shape)
     if n == 0:
         raise kv.KVSwapError(kv.kvswap_validate_shape(shape), "kvswap_workspace_bytes")
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    kv.kvswap_workspace_init(ws)
+    return ws
 
 
 def alloc_meta(shape: kv.kvswap_shape, device="cuda") -> torch.Tensor:

@@ -111,6 +111,7 @@ class DeviceLayer:
     def poison(self):
         """Fill every output and the workspace with NaN / garbage so unwritten results show."""
         self.ws.fill_(0xFF)
+        kv.kvswap_workspace_init(self.ws)
         self.meta.fill_(float("nan"))
         self.idx.fill_(-7)
         self.nsel.fill_(-7)

@@ -68,6 +68,7 @@ def run_layer_parity(li, scope):
     assert eo <= OUT_ATOL_TIGHT[wl.kv_dtype] and el <= OUT_ATOL_TIGHT[wl.kv_dtype], (eo, el)
     out2, _ = dl.sparse_decode(with_lse=False)
     assert np.array_equal(out, out2)                                       # deterministic, lse optional
+    assert kv.kvswap_read_device_status(dl.ws) == 0                        # no kernel gave up a wait
     return dl
 
 
