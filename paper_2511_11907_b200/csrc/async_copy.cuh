@@ -11,7 +11,7 @@
 
 namespace kvswap {
 
-constexpr uint32_t kWaitTries = 1u << 22;     // attempts per wait (each suspends briefly in hardware)
+constexpr uint32_t kWaitTries = 1u << 20;     // attempts per wait (each suspends briefly in hardware)
 
 // Device error words (written to the first word of the workspace, read by
 // kvswap_read_device_status).

@@ -8,17 +8,18 @@
 // which is cut into `splits` contiguous ranges, one CTA each, and every range into chunks of
 // kTok tokens.  A CTA serves RH query heads that share the KV head, so each K/V row is read once.
 //
-// CTA = kConsumers compute warps + 1 producer warp.  The producer resolves the token rows of a
-// chunk and brings their K and V rows into a ring of shared-memory stages with bulk asynchronous
-// copies (one copy per run of consecutive rows: a whole group when rows are dense), each stage
-// guarded by a full/empty mbarrier pair.  Chunk c belongs to consumer warp c % kConsumers, which
-// owns `depth` stages of the ring, so several chunks per warp are in flight while it computes.
+// Every warp of the CTA works alone on the chunks c = warp, warp + kWarps, ...: it owns `depth`
+// shared-memory stages, each guarded by an mbarrier, and keeps them filled itself.  Lanes 0..7
+// resolve the kTok token rows of a chunk and bring their K and V rows in with bulk asynchronous
+// copies (one copy per run of consecutive rows: a whole group when rows are dense); the copy for
+// chunk k + depth is issued the moment chunk k has been consumed, so `depth` chunks per warp are
+// in flight while it computes and no warp ever waits for another.
 //
-// A consumer warp owns D/32 channels per lane.  For a chunk it forms the kTok x RH partial dot
-// products of its channel slice, then transposes-and-sums them across the warp (a reduce-scatter
-// by shuffles) so that lane L ends up with the complete logit of (token L/4, head L%4): the
-// softmax bookkeeping then runs once per chunk with all 32 lanes busy.  Probabilities go through
-// a small shared-memory tile back to all lanes for the P.V update of their channel slice.
+// A warp owns D/32 channels per lane.  For a chunk it forms the kTok x RH partial dot products
+// of its channel slice, then transposes-and-sums them across the warp (a reduce-scatter by
+// shuffles) so that lane L ends up with the complete logit of (token L/4, head L%4): the softmax
+// bookkeeping then runs once per chunk with all 32 lanes busy.  Probabilities go through a small
+// shared-memory tile back to all lanes for the P.V update of their channel slice.
 #include <algorithm>
 
 #include "async_copy.cuh"
@@ -28,23 +29,20 @@ namespace kvswap {
 namespace {
 
 constexpr int kTok = 8;                         // tokens per stage
-constexpr int kConsumers = 8;                   // compute warps per CTA
-constexpr int kThreads = (kConsumers + 1) * 32;
-constexpr int kMaxDepth = 4;                    // stages per compute warp, at most
-constexpr int kMaxStages = kConsumers * kMaxDepth;
-constexpr int kIdxWindow = 1024;                // group indices the producer keeps on chip
+constexpr int kWarps = 8;                       // warps per CTA
+constexpr int kThreads = kWarps * 32;
+constexpr int kMaxDepth = 4;                    // stages per warp, at most
+constexpr int kMaxStages = kWarps * kMaxDepth;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 // Control block at the start of dynamic shared memory.
 struct Control {
   unsigned long long full[kMaxStages];          // data of the stage has landed
-  unsigned long long empty[kMaxStages];         // the stage may be overwritten
   uint32_t mask[kMaxStages];                    // bit t: token slot t of the stage holds a row
-  float prob[kConsumers][kTok * 4];             // softmax weights of the chunk, [token][head]
-  float corr[kConsumers][4];                    // rescale of the running accumulator, [head]
-  int32_t idx[kIdxWindow];                      // window of the selection list
-  volatile uint32_t abort;                      // a wait timed out somewhere in the CTA
+  float prob[kWarps][kTok * 4];                 // softmax weights of the chunk, [token][head]
+  float corr[kWarps][4];                        // rescale of the running accumulator, [head]
+  uint32_t abort;                               // a wait timed out somewhere in the CTA
 };
 constexpr int kControlBytes = (sizeof(Control) + 255) & ~255;
 
@@ -86,12 +84,23 @@ __device__ __forceinline__ void lds_row(uint32_t addr, float (&f)[DPL]) {
   }
 }
 
+// Where the attended tokens of one CTA come from.
+struct TokenSource {
+  const int32_t* idx;      // selection row
+  int NG, G, g_shift;      // g_shift = log2(G) when G is a power of two, else -1
+  int sel_tokens, tail0;   // n_sel * G, NG * G
+  int v_begin, v_end;      // this CTA's range of the virtual token list
+
+  // Group ordinal of virtual token v (v < sel_tokens).
+  __device__ __forceinline__ int group_of(int v) const { return g_shift >= 0 ? (v >> g_shift) : (v / G); }
+};
+
 template <typename KV_T, typename Q_T, int D, int RH>
 __global__ void __launch_bounds__(kThreads, 2)
 sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __restrict__ K,
                             const KV_T* __restrict__ V, const int32_t* __restrict__ group_idx,
                             const int32_t* __restrict__ n_selected, float* __restrict__ partial,
-                            int splits, int depth, uint32_t* __restrict__ err) {
+                            int splits, int depth, int g_shift, uint32_t* __restrict__ err) {
   constexpr int DPL = D / 32;                                  // channels per lane
   constexpr uint32_t ROWB = D * sizeof(KV_T);                  // bytes of one K or V row
   constexpr uint32_t HALFB = kTok * ROWB;                      // K (or V) part of a stage
@@ -103,7 +112,6 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   // Stage ring, aligned to HALFB so that a row index can be xor-ed into an address.
   const uint32_t ring = (smem_addr(smem_raw) + kControlBytes + HALFB - 1) & ~(HALFB - 1);
   unsigned char* ring_ptr = smem_raw + (ring - smem_addr(smem_raw));
-  const int n_stages = kConsumers * depth;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x;
@@ -114,10 +122,7 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   const int srow = (p.scope == KVSWAP_SCOPE_KV_HEAD) ? g : 0;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < n_stages; ++s) {
-      mbar_init(smem_addr(&ctl->full[s]), 1);
-      mbar_init(smem_addr(&ctl->empty[s]), 1);
-    }
+    for (int s = 0; s < kWarps * depth; ++s) mbar_init(smem_addr(&ctl->full[s]), 1);
     ctl->abort = 0;
     mbar_init_fence();
   }
@@ -127,15 +132,82 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   pdl_wait();
   pdl_trigger();
 
-  int n_sel = n_selected[int64_t(b) * p.S + srow];
-  n_sel = max(0, min(n_sel, p.M));
-  const int tail0 = p.NG * p.G;
-  const int sel_tokens = n_sel * p.G;
-  const int total = sel_tokens + (p.N - tail0);
-  int per_split = (total + splits - 1) / splits;
-  per_split = (per_split + kTok - 1) / kTok * kTok;
-  const int v_begin = min(total, per_split * split), v_end = min(total, v_begin + per_split);
-  const int n_chunks = (v_end - v_begin + kTok - 1) / kTok;
+  TokenSource src;
+  src.idx = group_idx + (int64_t(b) * p.S + srow) * p.M;
+  src.NG = p.NG; src.G = p.G; src.g_shift = g_shift;
+  {
+    int n_sel = n_selected[int64_t(b) * p.S + srow];
+    n_sel = max(0, min(n_sel, p.M));
+    src.tail0 = p.NG * p.G;
+    src.sel_tokens = n_sel * p.G;
+    const int total = src.sel_tokens + (p.N - src.tail0);
+    int per_split = (total + splits - 1) / splits;
+    per_split = (per_split + kTok - 1) / kTok * kTok;
+    src.v_begin = min(total, per_split * split);
+    src.v_end = min(total, src.v_begin + per_split);
+  }
+  const int n_chunks = (src.v_end - src.v_begin + kTok - 1) / kTok;
+  const int my_chunks = (n_chunks > warp) ? (n_chunks - warp + kWarps - 1) / kWarps : 0;   // of this warp
+
+  const KV_T* Kg = K + int64_t(b) * p.kv_sb + int64_t(g) * p.kv_sh;
+  const KV_T* Vg = V + int64_t(b) * p.kv_sb + int64_t(g) * p.kv_sh;
+  const bool dense = (p.kv_sn == D);
+
+  // Group index (or -1) behind token slot `lane` of this warp's k-th chunk: the one global read
+  // of the fill path, issued early so that its latency hides behind the compute of a chunk.
+  auto fetch_group = [&](int k) -> int {
+    const int v = src.v_begin + (warp + k * kWarps) * kTok + lane;
+    if (lane < kTok && k < my_chunks && v < src.v_end && v < src.sel_tokens) return src.idx[src.group_of(v)];
+    return -1;
+  };
+  // Fill: bring chunk k into `stage`.  `j` is fetch_group(k).  All 32 lanes call.
+  auto fill = [&](int k, int j, int stage) {
+    const int v = src.v_begin + (warp + k * kWarps) * kTok + lane;
+    int n = -1;
+    if (lane < kTok && v < src.v_end) {
+      if (v < src.sel_tokens) {
+        if (j >= 0 && j < src.NG) n = j * src.G + (v - src.group_of(v) * src.G);
+      } else {
+        n = src.tail0 + (v - src.sel_tokens);
+      }
+    }
+    const bool valid = n >= 0;
+    const uint32_t vmask = __ballot_sync(kFull, valid);
+    const int n_prev = __shfl_up_sync(kFull, n, 1);
+    const bool head = valid && (!dense || lane == 0 || !((vmask >> (lane - 1)) & 1u) || n != n_prev + 1);
+    const uint32_t heads = __ballot_sync(kFull, head);
+    const uint32_t bar = smem_addr(&ctl->full[stage]);
+    if (lane == 0) {
+      ctl->mask[stage] = vmask;
+      mbar_arrive_expect_tx(bar, uint32_t(__popc(vmask)) * 2u * ROWB);
+    }
+    if (head) {
+      const uint32_t stop = (heads | ~vmask | (1u << kTok)) & ~((2u << lane) - 1u);
+      const uint32_t run = uint32_t(__ffs(int(stop)) - 1 - lane);
+      const uint32_t dst = ring + uint32_t(stage) * STAGEB + uint32_t(lane) * ROWB;
+      bulk_g2s(dst, Kg + int64_t(n) * p.kv_sn, run * ROWB, bar);
+      bulk_g2s(dst + HALFB, Vg + int64_t(n) * p.kv_sn, run * ROWB, bar);
+    }
+  };
+
+  // ---- prologue: fill the first `depth` stages ---------------------------------------------------
+  {
+    int j0[kMaxDepth];
+#pragma unroll
+    for (int k = 0; k < kMaxDepth; ++k) j0[k] = (k < depth) ? fetch_group(k) : -1;
+#pragma unroll
+    for (int k = 0; k < kMaxDepth; ++k)
+      if (k < depth && k < my_chunks) fill(k, j0[k], warp + kWarps * k);
+  }
+
+  // q slice of this lane, pre-scaled by log2(e)/sqrt(d): logits live in the log2 domain.
+  const float scale = kLog2e * rsqrtf(float(D));
+  float qr[RH][DPL];
+#pragma unroll
+  for (int hh = 0; hh < RH; ++hh)
+#pragma unroll
+    for (int j = 0; j < DPL; ++j)
+      qr[hh][j] = q_to_float(q[(int64_t(b) * p.Hq + h0 + hh) * D + lane * DPL + j]) * scale;
 
   float m_run = -INFINITY, l_run = 0.f;           // of head lane % 4 (replicated over the tokens)
   float acc[RH][DPL];
@@ -144,256 +216,135 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
 #pragma unroll
     for (int j = 0; j < DPL; ++j) acc[hh][j] = 0.f;
 
-  if (warp == kConsumers) {
-    // ================================ producer ==============================================
-    const int32_t* idx = group_idx + (int64_t(b) * p.S + srow) * p.M;
-    const KV_T* Kg = K + int64_t(b) * p.kv_sb + int64_t(g) * p.kv_sh;
-    const KV_T* Vg = V + int64_t(b) * p.kv_sb + int64_t(g) * p.kv_sh;
-    const bool dense = (p.kv_sn == D);
-    if (dense && p.G % kTok == 0) {
-      // ---- whole chunks: a chunk is kTok consecutive rows of one group (or of the tail), so one
-      // lane resolves and issues one chunk.  An iteration covers every stage of the ring once:
-      // chunk it * n_stages + lane lives in stage `lane` and is its use number `it`.
-      for (int it = 0, base = 0; base < n_chunks; ++it, base += n_stages) {
-        const int cl = base + lane;
-        bool ok = true;
-        if (lane < n_stages && cl < n_chunks) {
-          if (it > 0) ok = mbar_wait(smem_addr(&ctl->empty[lane]), uint32_t(it - 1) & 1u);
-          if (ok) {
-            const int v = v_begin + cl * kTok;
-            const int rows = min(kTok, v_end - v);
-            int n = -1;
-            if (v < sel_tokens) {
-              const int go = v / p.G;
-              const int j = idx[go];
-              if (j >= 0 && j < p.NG) n = j * p.G + (v - go * p.G);
-            } else {
-              n = tail0 + (v - sel_tokens);
-            }
-            const uint32_t bar = smem_addr(&ctl->full[lane]);
-            ctl->mask[lane] = (n >= 0) ? ((1u << rows) - 1u) : 0u;
-            mbar_arrive_expect_tx(bar, (n >= 0) ? uint32_t(rows) * 2u * ROWB : 0u);
-            if (n >= 0) {
-              const uint32_t dst = ring + uint32_t(lane) * STAGEB;
-              bulk_g2s(dst, Kg + int64_t(n) * p.kv_sn, uint32_t(rows) * ROWB, bar);
-              bulk_g2s(dst + HALFB, Vg + int64_t(n) * p.kv_sn, uint32_t(rows) * ROWB, bar);
-            }
+  const int tok = lane >> 2, hd = lane & 3;        // the (token, head) this lane finishes
+  const uint32_t lane_off = uint32_t(lane) * DPL * sizeof(KV_T);
+  const uint32_t xperm = uint32_t(tok) * ROWB;     // slot s of this lane holds token s ^ tok
+  float* prob = ctl->prob[warp];
+  float* corr = ctl->corr[warp];
+  int slot = 0;
+  uint32_t phase = 0;
+  bool timed_out = false;
+  for (int k = 0; k < my_chunks; ++k) {
+    const int stage = warp + kWarps * slot;
+    const int j_next = fetch_group(k + depth);     // consumed by the refill at the end of the iteration
+    if (!__all_sync(kFull, mbar_wait(smem_addr(&ctl->full[stage]), phase))) { timed_out = true; break; }
+    const uint32_t mask = ctl->mask[stage];
+    if (mask != 0u) {
+      const uint32_t kbase = (ring + uint32_t(stage) * STAGEB + lane_off) ^ xperm;
+      const uint32_t vbase = ring + uint32_t(stage) * STAGEB + HALFB + lane_off;
+
+      // ---- partial q.k of this lane's channels: slot s <-> token s ^ tok ---------------------
+      float part[kTok][4];
+#pragma unroll
+      for (int s = 0; s < kTok; ++s) {
+        float kf[DPL];
+        lds_row<KV_T, DPL>(kbase ^ (uint32_t(s) * ROWB), kf);
+#pragma unroll
+        for (int hh = 0; hh < 4; ++hh) {
+          float a = 0.f;
+          if (hh < RH) {
+#pragma unroll
+            for (int j = 0; j < DPL; ++j) a = fmaf(qr[hh][j], kf[j], a);
           }
+          part[s][hh] = a;
         }
-        if (!__all_sync(kFull, ok)) {
-          if (lane == 0) { ctl->abort = 1; if (err) atomicExch(err, kDevTimeoutEmpty); }
-          break;
-        }
-        if (__any_sync(kFull, ctl->abort != 0u)) break;
       }
-    } else {
-      // ---- any group size or row stride: four chunks per iteration, one lane per token row;
-      // runs of consecutive rows share a copy.  Lane = 8 * (chunk in the batch) + token slot.
-      constexpr int kBatch = 32 / kTok;
-      const int cb = lane / kTok, t = lane % kTok;
-      int win_base = 0, win_len = 0;
-      int cw = 0, slot = 0, use = 0;              // stage (cw + cb, slot) is on its use number `use`
-      for (int cl = 0; cl < n_chunks; cl += kBatch) {
-        const int stage = cw + cb + kConsumers * slot;
-        const bool active = cl + cb < n_chunks;
-        bool ok = true;
-        if (active && use > 0) ok = mbar_wait(smem_addr(&ctl->empty[stage]), uint32_t(use - 1) & 1u);
-        if (!__all_sync(kFull, ok)) {
-          if (lane == 0) { ctl->abort = 1; if (err) atomicExch(err, kDevTimeoutEmpty); }
-          break;
+      // ---- reduce-scatter over the warp: tokens over lane bits 4..2, heads over bits 1..0 ------
+#pragma unroll
+      for (int s = 0; s < 4; ++s)
+#pragma unroll
+        for (int hh = 0; hh < RH; ++hh) part[s][hh] += __shfl_xor_sync(kFull, part[s + 4][hh], 16);
+#pragma unroll
+      for (int s = 0; s < 2; ++s)
+#pragma unroll
+        for (int hh = 0; hh < RH; ++hh) part[s][hh] += __shfl_xor_sync(kFull, part[s + 2][hh], 8);
+#pragma unroll
+      for (int hh = 0; hh < RH; ++hh) part[0][hh] += __shfl_xor_sync(kFull, part[1][hh], 4);
+      const bool b1 = lane & 2, b0 = lane & 1;
+      const float keep0 = b1 ? part[0][2] : part[0][0], keep1 = b1 ? part[0][3] : part[0][1];
+      const float send0 = b1 ? part[0][0] : part[0][2], send1 = b1 ? part[0][1] : part[0][3];
+      const float r0 = keep0 + __shfl_xor_sync(kFull, send0, 2);
+      const float r1 = keep1 + __shfl_xor_sync(kFull, send1, 2);
+      float s_log = (b0 ? r1 : r0) + __shfl_xor_sync(kFull, b0 ? r0 : r1, 1);
+
+      // ---- online softmax for (token tok, head hd) ----------------------------------------------
+      const bool live = ((mask >> tok) & 1u) && hd < RH;
+      s_log = live ? s_log : -INFINITY;
+      float cmax = s_log;
+      cmax = fmaxf(cmax, __shfl_xor_sync(kFull, cmax, 4));
+      cmax = fmaxf(cmax, __shfl_xor_sync(kFull, cmax, 8));
+      cmax = fmaxf(cmax, __shfl_xor_sync(kFull, cmax, 16));
+      const float m_new = fmaxf(m_run, cmax);
+      const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+      const float pw = ex2(s_log - m_safe);          // 0 for dead (token, head) pairs
+      const float cr = ex2(m_run - m_safe);          // 0 while nothing has been seen yet
+      float psum = pw;
+      psum += __shfl_xor_sync(kFull, psum, 4);
+      psum += __shfl_xor_sync(kFull, psum, 8);
+      psum += __shfl_xor_sync(kFull, psum, 16);
+      l_run = fmaf(l_run, cr, psum);
+      m_run = m_new;
+      prob[lane] = pw;
+      if (tok == 0) corr[hd] = cr;
+      __syncwarp();
+
+      // ---- P.V on this lane's channels -----------------------------------------------------------
+      const float4 c4 = *reinterpret_cast<const float4*>(corr);
+      const float cv[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+      for (int hh = 0; hh < RH; ++hh)
+#pragma unroll
+        for (int j = 0; j < DPL; ++j) acc[hh][j] *= cv[hh];
+#pragma unroll
+      for (int t = 0; t < kTok; ++t) {
+        if ((mask >> t) & 1u) {                     // warp-uniform; stale rows are never read
+          float vf[DPL];
+          lds_row<KV_T, DPL>(vbase + uint32_t(t) * ROWB, vf);
+          const float4 p4 = *reinterpret_cast<const float4*>(prob + 4 * t);
+          const float pv[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+          for (int hh = 0; hh < RH; ++hh)
+#pragma unroll
+            for (int j = 0; j < DPL; ++j) acc[hh][j] = fmaf(pv[hh], vf[j], acc[hh][j]);
         }
-        if (__any_sync(kFull, ctl->abort != 0u)) break;
-        const int v0 = v_begin + cl * kTok;
-        // refill the index window if this batch reaches beyond it (warp-uniform)
-        if (v0 < sel_tokens) {
-          const int go_first = v0 / p.G;
-          const int go_last = (min(min(v0 + 32, v_end), sel_tokens) - 1) / p.G;
-          if (go_first < win_base || go_last >= win_base + win_len) {
-            __syncwarp();
-            win_base = go_first;
-            win_len = min(kIdxWindow, n_sel - win_base);
-            for (int i = lane; i < win_len; i += 32) ctl->idx[i] = idx[win_base + i];
-            __syncwarp();
-          }
-        }
-        const int v = v0 + lane;
-        int n = -1;
-        if (v < v_end) {
-          if (v < sel_tokens) {
-            const int go = v / p.G;
-            const int j = ctl->idx[go - win_base];
-            if (j >= 0 && j < p.NG) n = j * p.G + (v - go * p.G);
-          } else {
-            n = tail0 + (v - sel_tokens);
-          }
-        }
-        const bool valid = n >= 0;
-        const uint32_t vmask = (__ballot_sync(kFull, valid) >> (cb * kTok)) & ((1u << kTok) - 1u);
-        const int n_prev = __shfl_up_sync(kFull, n, 1);
-        const bool head = valid && (!dense || t == 0 || !((vmask >> (t - 1)) & 1u) || n != n_prev + 1);
-        const uint32_t heads = (__ballot_sync(kFull, head) >> (cb * kTok)) & ((1u << kTok) - 1u);
-        const uint32_t bar = smem_addr(&ctl->full[stage]);
-        if (active && t == 0) {
-          ctl->mask[stage] = vmask;
-          mbar_arrive_expect_tx(bar, uint32_t(__popc(vmask)) * 2u * ROWB);
-        }
-        if (head) {
-          const uint32_t stop = (heads | ~vmask | (1u << kTok)) & ~((2u << t) - 1u);
-          const uint32_t run = uint32_t(__ffs(int(stop)) - 1 - t);
-          const uint32_t dst = ring + uint32_t(stage) * STAGEB + uint32_t(t) * ROWB;
-          bulk_g2s(dst, Kg + int64_t(n) * p.kv_sn, run * ROWB, bar);
-          bulk_g2s(dst + HALFB, Vg + int64_t(n) * p.kv_sn, run * ROWB, bar);
-        }
-        cw += kBatch;
-        if (cw == kConsumers) { cw = 0; if (++slot == depth) { slot = 0; ++use; } }
       }
     }
-  } else {
-    // ================================ consumers =============================================
-    // q slice of this lane, pre-scaled by log2(e)/sqrt(d): logits live in the log2 domain.
-    const float scale = kLog2e * rsqrtf(float(D));
-    float qr[RH][DPL];
-#pragma unroll
-    for (int hh = 0; hh < RH; ++hh)
-#pragma unroll
-      for (int j = 0; j < DPL; ++j)
-        qr[hh][j] = q_to_float(q[(int64_t(b) * p.Hq + h0 + hh) * D + lane * DPL + j]) * scale;
-
-    const int tok = lane >> 2, hd = lane & 3;      // the (token, head) this lane finishes
-    const uint32_t lane_off = uint32_t(lane) * DPL * sizeof(KV_T);
-    const uint32_t xperm = uint32_t(tok) * ROWB;   // slot s of this lane holds token s ^ tok
-    float* prob = ctl->prob[warp];
-    float* corr = ctl->corr[warp];
-    int slot = 0;
-    uint32_t phase = 0;
-    for (int cl = warp; cl < n_chunks; cl += kConsumers) {
-      const int stage = warp + kConsumers * slot;
-      if (__any_sync(kFull, ctl->abort != 0u)) break;
-      if (!__all_sync(kFull, mbar_wait(smem_addr(&ctl->full[stage]), phase))) {
-        if (lane == 0) { ctl->abort = 1; if (err) atomicExch(err, kDevTimeoutFull); }
-        break;
-      }
-      const uint32_t mask = ctl->mask[stage];
-      if (mask != 0u) {
-        const uint32_t kbase = (ring + uint32_t(stage) * STAGEB + lane_off) ^ xperm;
-        const uint32_t vbase = ring + uint32_t(stage) * STAGEB + HALFB + lane_off;
-
-        // ---- partial q.k of this lane's channels: slot s <-> token s ^ tok -----------------
-        float part[kTok][4];
-#pragma unroll
-        for (int s = 0; s < kTok; ++s) {
-          float kf[DPL];
-          lds_row<KV_T, DPL>(kbase ^ (uint32_t(s) * ROWB), kf);
-#pragma unroll
-          for (int hh = 0; hh < 4; ++hh) {
-            float a = 0.f;
-            if (hh < RH) {
-#pragma unroll
-              for (int j = 0; j < DPL; ++j) a = fmaf(qr[hh][j], kf[j], a);
-            }
-            part[s][hh] = a;
-          }
-        }
-        // ---- reduce-scatter over the warp: tokens over lane bits 4..2, heads over bits 1..0 ---
-#pragma unroll
-        for (int s = 0; s < 4; ++s)
-#pragma unroll
-          for (int hh = 0; hh < RH; ++hh) part[s][hh] += __shfl_xor_sync(kFull, part[s + 4][hh], 16);
-#pragma unroll
-        for (int s = 0; s < 2; ++s)
-#pragma unroll
-          for (int hh = 0; hh < RH; ++hh) part[s][hh] += __shfl_xor_sync(kFull, part[s + 2][hh], 8);
-#pragma unroll
-        for (int hh = 0; hh < RH; ++hh) part[0][hh] += __shfl_xor_sync(kFull, part[1][hh], 4);
-        const bool b1 = lane & 2, b0 = lane & 1;
-        const float keep0 = b1 ? part[0][2] : part[0][0], keep1 = b1 ? part[0][3] : part[0][1];
-        const float send0 = b1 ? part[0][0] : part[0][2], send1 = b1 ? part[0][1] : part[0][3];
-        const float r0 = keep0 + __shfl_xor_sync(kFull, send0, 2);
-        const float r1 = keep1 + __shfl_xor_sync(kFull, send1, 2);
-        float s_log = (b0 ? r1 : r0) + __shfl_xor_sync(kFull, b0 ? r0 : r1, 1);
-
-        // ---- online softmax for (token tok, head hd) ------------------------------------------
-        const bool live = ((mask >> tok) & 1u) && hd < RH;
-        s_log = live ? s_log : -INFINITY;
-        float cmax = s_log;
-        cmax = fmaxf(cmax, __shfl_xor_sync(kFull, cmax, 4));
-        cmax = fmaxf(cmax, __shfl_xor_sync(kFull, cmax, 8));
-        cmax = fmaxf(cmax, __shfl_xor_sync(kFull, cmax, 16));
-        const float m_new = fmaxf(m_run, cmax);
-        const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-        const float pw = ex2(s_log - m_safe);          // 0 for dead (token, head) pairs
-        const float cr = ex2(m_run - m_safe);          // 0 while nothing has been seen yet
-        float psum = pw;
-        psum += __shfl_xor_sync(kFull, psum, 4);
-        psum += __shfl_xor_sync(kFull, psum, 8);
-        psum += __shfl_xor_sync(kFull, psum, 16);
-        l_run = fmaf(l_run, cr, psum);
-        m_run = m_new;
-        prob[lane] = pw;
-        if (tok == 0) corr[hd] = cr;
-        __syncwarp();
-
-        // ---- P.V on this lane's channels -------------------------------------------------------
-        const float4 c4 = *reinterpret_cast<const float4*>(corr);
-        const float cv[4] = {c4.x, c4.y, c4.z, c4.w};
-#pragma unroll
-        for (int hh = 0; hh < RH; ++hh)
-#pragma unroll
-          for (int j = 0; j < DPL; ++j) acc[hh][j] *= cv[hh];
-#pragma unroll
-        for (int t = 0; t < kTok; ++t) {
-          if ((mask >> t) & 1u) {                     // warp-uniform; stale rows are never read
-            float vf[DPL];
-            lds_row<KV_T, DPL>(vbase + uint32_t(t) * ROWB, vf);
-            const float4 p4 = *reinterpret_cast<const float4*>(prob + 4 * t);
-            const float pv[4] = {p4.x, p4.y, p4.z, p4.w};
-#pragma unroll
-            for (int hh = 0; hh < RH; ++hh)
-#pragma unroll
-              for (int j = 0; j < DPL; ++j) acc[hh][j] = fmaf(pv[hh], vf[j], acc[hh][j]);
-          }
-        }
-      }
-      __syncwarp();                                   // all lanes are done with the stage and prob[]
-      if (lane == 0) mbar_arrive(smem_addr(&ctl->empty[stage]));
-      if (++slot == depth) { slot = 0; phase ^= 1u; }
+    __syncwarp();                                   // all lanes are done with the stage and prob[]
+    if (k + depth < my_chunks) fill(k + depth, j_next, stage);
+    if (++slot == depth) { slot = 0; phase ^= 1u; }
+  }
+  if (timed_out) {
+    // The wait gave up: record it, and before the CTA's shared memory is released give this
+    // warp's copies that may still be in flight a bounded chance to land.  The partial written
+    // below is then meaningless; the status word tells the host.
+    if (lane == 0) { ctl->abort = 1; if (err) atomicExch(err, kDevTimeoutFull); }
+    for (int s = 0; s < depth; ++s) {
+      mbar_wait(smem_addr(&ctl->full[warp + kWarps * s]), 0);
+      mbar_wait(smem_addr(&ctl->full[warp + kWarps * s]), 1);
     }
   }
 
-  // ---- merge the compute warps of the CTA ------------------------------------------------------
+  // ---- merge the warps of the CTA ------------------------------------------------------------------
   __syncthreads();               // every loop above is bounded, so every warp arrives here
-  if (ctl->abort) {
-    // A wait gave up: before the CTA's shared memory is released, give copies that may still be
-    // in flight a bounded chance to land.  The partial written below is then meaningless; the
-    // error word tells the host.
-    if (threadIdx.x == 0)
-      for (int s = 0; s < n_stages; ++s) {
-        mbar_wait(smem_addr(&ctl->full[s]), 0);
-        mbar_wait(smem_addr(&ctl->full[s]), 1);
-      }
-    __syncthreads();
-  }
   // The ring is idle now (every issued copy was waited for); reuse it for the merge.
-  float* sm_m = reinterpret_cast<float*>(ring_ptr);                 // [kConsumers][4]
-  float* sm_l = sm_m + kConsumers * 4;                              // [kConsumers][4]
-  float* sm_acc = sm_l + kConsumers * 4;                            // [kConsumers][RH][D]
-  if (warp < kConsumers) {
-    if (lane < 4) { sm_m[warp * 4 + lane] = m_run; sm_l[warp * 4 + lane] = l_run; }
+  float* sm_m = reinterpret_cast<float*>(ring_ptr);                 // [kWarps][4]
+  float* sm_l = sm_m + kWarps * 4;                                  // [kWarps][4]
+  float* sm_acc = sm_l + kWarps * 4;                                // [kWarps][RH][D]
+  if (lane < 4) { sm_m[warp * 4 + lane] = m_run; sm_l[warp * 4 + lane] = l_run; }
 #pragma unroll
-    for (int hh = 0; hh < RH; ++hh)
+  for (int hh = 0; hh < RH; ++hh)
 #pragma unroll
-      for (int j = 0; j < DPL; ++j) sm_acc[(warp * RH + hh) * D + lane * DPL + j] = acc[hh][j];
-  }
+    for (int j = 0; j < DPL; ++j) sm_acc[(warp * RH + hh) * D + lane * DPL + j] = acc[hh][j];
   __syncthreads();
   for (int i = threadIdx.x; i < RH * D; i += kThreads) {
     const int hh = i / D, c = i % D;
     float mx = -INFINITY;
 #pragma unroll
-    for (int k = 0; k < kConsumers; ++k) mx = fmaxf(mx, sm_m[k * 4 + hh]);
+    for (int k = 0; k < kWarps; ++k) mx = fmaxf(mx, sm_m[k * 4 + hh]);
     float lsum = 0.f, a = 0.f;
     if (mx > -INFINITY) {
 #pragma unroll
-      for (int k = 0; k < kConsumers; ++k) {
+      for (int k = 0; k < kWarps; ++k) {
         const float w = ex2(sm_m[k * 4 + hh] - mx);
         lsum = fmaf(sm_l[k * 4 + hh], w, lsum);
         a = fmaf(sm_acc[(k * RH + hh) * D + c], w, a);
@@ -436,13 +387,15 @@ cudaError_t launch_one(const Problem& p, const Workspace& w, const void* q, cons
                        const int32_t* group_idx, const int32_t* n_selected, float* partial, float* out, float* lse,
                        uint32_t* err, cudaStream_t st) {
   const int depth = w.depth;
-  const size_t smem = kControlBytes + stage_bytes<KV_T, D>() / 2 + size_t(kConsumers) * depth * stage_bytes<KV_T, D>();
+  const size_t smem = kControlBytes + stage_bytes<KV_T, D>() / 2 + size_t(kWarps) * depth * stage_bytes<KV_T, D>();
+  int g_shift = -1;
+  for (int sft = 0; sft < 31; ++sft) if ((1 << sft) == p.G) g_shift = sft;
   auto kern = sparse_decode_splitk_kernel<KV_T, Q_T, D, RH>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
   if (e != cudaSuccess) return e;
   e = launch_pdl(kern, dim3(w.splits, p.Hkv * (p.rho / RH), p.B), dim3(kThreads), smem, st, p,
                  static_cast<const Q_T*>(q), static_cast<const KV_T*>(K), static_cast<const KV_T*>(V), group_idx,
-                 n_selected, partial, w.splits, depth, err);
+                 n_selected, partial, w.splits, depth, g_shift, err);
   if (e != cudaSuccess) return e;
   return launch_pdl(combine_kernel<D>, dim3(p.B * p.Hq), dim3(D), 0, st, static_cast<const float*>(partial), out,
                     lse, w.splits);
@@ -491,7 +444,7 @@ void plan_sparse_decode(const Problem& p, Workspace* w) {
   // One wave of 2 CTAs per SM when the problems are few; otherwise the split that fills whole
   // waves best, keeping at least two chunks per compute warp and split.
   const int64_t slots = int64_t(kNumSMs) * 2;
-  const int64_t max_splits = std::min<int64_t>(256, std::max<int64_t>(1, n_chunks / (2 * kConsumers)));
+  const int64_t max_splits = std::min<int64_t>(256, std::max<int64_t>(1, n_chunks / (2 * kWarps)));
   int64_t best = 1;
   double best_eff = 0.0;
   for (int64_t s = 1; s <= max_splits; ++s) {
@@ -505,7 +458,7 @@ void plan_sparse_decode(const Problem& p, Workspace* w) {
   w->splits = int(best);
   const size_t row = size_t(p.d) * (p.kv_dtype == KVSWAP_F32 ? 4 : 2);
   const size_t stage = 2 * kTok * row;
-  w->depth = int(std::max<size_t>(2, std::min<size_t>(kMaxDepth, (100u << 10) / (kConsumers * stage))));
+  w->depth = int(std::max<size_t>(2, std::min<size_t>(kMaxDepth, (100u << 10) / (kWarps * stage))));
 }
 
 cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K, const void* V,
