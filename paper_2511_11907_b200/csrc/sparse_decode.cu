@@ -40,8 +40,8 @@ constexpr float kLn2 = 0.6931471805599453f;
 struct Control {
   unsigned long long full[kMaxStages];          // data of the stage has landed
   uint32_t mask[kMaxStages];                    // bit t: token slot t of the stage holds a row
-  float prob[kWarps][kTok * 4];                 // softmax weights of the chunk, [token][head]
-  float corr[kWarps][4];                        // rescale of the running accumulator, [head]
+  float2 prob[kWarps][kTok * 4];                // softmax weights of the chunk, [token][head], each twice
+  float2 corr[kWarps][4];                       // rescale of the running accumulator, [head], each twice
   uint32_t abort;                               // a wait timed out somewhere in the CTA
 };
 constexpr int kControlBytes = (sizeof(Control) + 255) & ~255;
@@ -153,16 +153,41 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   const KV_T* Vg = V + int64_t(b) * p.kv_sb + int64_t(g) * p.kv_sh;
   const bool dense = (p.kv_sn == D);
 
+  // When rows are dense and G is a multiple of kTok, a chunk is kTok consecutive rows of one
+  // group (or of the tail): lane 0 alone resolves it and issues one copy each for K and V.
+  const bool whole = dense && (p.G % kTok == 0);
+
   // Group index (or -1) behind token slot `lane` of this warp's k-th chunk: the one global read
   // of the fill path, issued early so that its latency hides behind the compute of a chunk.
   auto fetch_group = [&](int k) -> int {
     const int v = src.v_begin + (warp + k * kWarps) * kTok + lane;
-    if (lane < kTok && k < my_chunks && v < src.v_end && v < src.sel_tokens) return src.idx[src.group_of(v)];
+    if (lane < (whole ? 1 : kTok) && k < my_chunks && v < src.v_end && v < src.sel_tokens)
+      return src.idx[src.group_of(v)];
     return -1;
   };
   // Fill: bring chunk k into `stage`.  `j` is fetch_group(k).  All 32 lanes call.
   auto fill = [&](int k, int j, int stage) {
     const int v = src.v_begin + (warp + k * kWarps) * kTok + lane;
+    const uint32_t bar = smem_addr(&ctl->full[stage]);
+    if (whole) {
+      if (lane == 0) {
+        const int rows = min(kTok, src.v_end - v);
+        int n = -1;
+        if (v < src.sel_tokens) {
+          if (j >= 0 && j < src.NG) n = j * src.G + (v - src.group_of(v) * src.G);
+        } else {
+          n = src.tail0 + (v - src.sel_tokens);
+        }
+        ctl->mask[stage] = (n >= 0) ? ((1u << rows) - 1u) : 0u;
+        mbar_arrive_expect_tx(bar, (n >= 0) ? uint32_t(rows) * 2u * ROWB : 0u);
+        if (n >= 0) {
+          const uint32_t dst = ring + uint32_t(stage) * STAGEB;
+          bulk_g2s(dst, Kg + int64_t(n) * D, uint32_t(rows) * ROWB, bar);
+          bulk_g2s(dst + HALFB, Vg + int64_t(n) * D, uint32_t(rows) * ROWB, bar);
+        }
+      }
+      return;
+    }
     int n = -1;
     if (lane < kTok && v < src.v_end) {
       if (v < src.sel_tokens) {
@@ -176,7 +201,6 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
     const int n_prev = __shfl_up_sync(kFull, n, 1);
     const bool head = valid && (!dense || lane == 0 || !((vmask >> (lane - 1)) & 1u) || n != n_prev + 1);
     const uint32_t heads = __ballot_sync(kFull, head);
-    const uint32_t bar = smem_addr(&ctl->full[stage]);
     if (lane == 0) {
       ctl->mask[stage] = vmask;
       mbar_arrive_expect_tx(bar, uint32_t(__popc(vmask)) * 2u * ROWB);
@@ -200,27 +224,30 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
       if (k < depth && k < my_chunks) fill(k, j0[k], warp + kWarps * k);
   }
 
-  // q slice of this lane, pre-scaled by log2(e)/sqrt(d): logits live in the log2 domain.
+  // q slice of this lane, pre-scaled by log2(e)/sqrt(d) (logits live in the log2 domain), each
+  // value twice: the packed FMA below works on two tokens at a time.
   const float scale = kLog2e * rsqrtf(float(D));
-  float qr[RH][DPL];
+  float2 qq[RH][DPL];
 #pragma unroll
   for (int hh = 0; hh < RH; ++hh)
 #pragma unroll
-    for (int j = 0; j < DPL; ++j)
-      qr[hh][j] = q_to_float(q[(int64_t(b) * p.Hq + h0 + hh) * D + lane * DPL + j]) * scale;
+    for (int j = 0; j < DPL; ++j) {
+      const float x = q_to_float(q[(int64_t(b) * p.Hq + h0 + hh) * D + lane * DPL + j]) * scale;
+      qq[hh][j] = make_float2(x, x);
+    }
 
   float m_run = -INFINITY, l_run = 0.f;           // of head lane % 4 (replicated over the tokens)
-  float acc[RH][DPL];
+  float2 acc[RH][DPL / 2];                         // channel pairs
 #pragma unroll
   for (int hh = 0; hh < RH; ++hh)
 #pragma unroll
-    for (int j = 0; j < DPL; ++j) acc[hh][j] = 0.f;
+    for (int j = 0; j < DPL / 2; ++j) acc[hh][j] = make_float2(0.f, 0.f);
 
   const int tok = lane >> 2, hd = lane & 3;        // the (token, head) this lane finishes
   const uint32_t lane_off = uint32_t(lane) * DPL * sizeof(KV_T);
   const uint32_t xperm = uint32_t(tok) * ROWB;     // slot s of this lane holds token s ^ tok
-  float* prob = ctl->prob[warp];
-  float* corr = ctl->corr[warp];
+  float2* prob = ctl->prob[warp];
+  float2* corr = ctl->corr[warp];
   int slot = 0;
   uint32_t phase = 0;
   bool timed_out = false;
@@ -233,36 +260,41 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
       const uint32_t kbase = (ring + uint32_t(stage) * STAGEB + lane_off) ^ xperm;
       const uint32_t vbase = ring + uint32_t(stage) * STAGEB + HALFB + lane_off;
 
-      // ---- partial q.k of this lane's channels: slot s <-> token s ^ tok ---------------------
-      float part[kTok][4];
+      // ---- partial q.k of this lane's channels; slot s <-> token s ^ tok, slots s and s + 4 share
+      // a packed accumulator (.x, .y) ------------------------------------------------------------
+      float2 part[4][4];
 #pragma unroll
-      for (int s = 0; s < kTok; ++s) {
-        float kf[DPL];
-        lds_row<KV_T, DPL>(kbase ^ (uint32_t(s) * ROWB), kf);
+      for (int s = 0; s < 4; ++s) {
+        float ka[DPL], kb[DPL];
+        lds_row<KV_T, DPL>(kbase ^ (uint32_t(s) * ROWB), ka);
+        lds_row<KV_T, DPL>(kbase ^ (uint32_t(s + 4) * ROWB), kb);
 #pragma unroll
         for (int hh = 0; hh < 4; ++hh) {
-          float a = 0.f;
+          float2 a = make_float2(0.f, 0.f);
           if (hh < RH) {
+            a = __fmul2_rn(qq[hh][0], make_float2(ka[0], kb[0]));
 #pragma unroll
-            for (int j = 0; j < DPL; ++j) a = fmaf(qr[hh][j], kf[j], a);
+            for (int j = 1; j < DPL; ++j) a = __ffma2_rn(qq[hh][j], make_float2(ka[j], kb[j]), a);
           }
           part[s][hh] = a;
         }
       }
       // ---- reduce-scatter over the warp: tokens over lane bits 4..2, heads over bits 1..0 ------
+      float red[4][4];
 #pragma unroll
       for (int s = 0; s < 4; ++s)
 #pragma unroll
-        for (int hh = 0; hh < RH; ++hh) part[s][hh] += __shfl_xor_sync(kFull, part[s + 4][hh], 16);
+        for (int hh = 0; hh < 4; ++hh)
+          red[s][hh] = (hh < RH) ? part[s][hh].x + __shfl_xor_sync(kFull, part[s][hh].y, 16) : 0.f;
 #pragma unroll
       for (int s = 0; s < 2; ++s)
 #pragma unroll
-        for (int hh = 0; hh < RH; ++hh) part[s][hh] += __shfl_xor_sync(kFull, part[s + 2][hh], 8);
+        for (int hh = 0; hh < RH; ++hh) red[s][hh] += __shfl_xor_sync(kFull, red[s + 2][hh], 8);
 #pragma unroll
-      for (int hh = 0; hh < RH; ++hh) part[0][hh] += __shfl_xor_sync(kFull, part[1][hh], 4);
+      for (int hh = 0; hh < RH; ++hh) red[0][hh] += __shfl_xor_sync(kFull, red[1][hh], 4);
       const bool b1 = lane & 2, b0 = lane & 1;
-      const float keep0 = b1 ? part[0][2] : part[0][0], keep1 = b1 ? part[0][3] : part[0][1];
-      const float send0 = b1 ? part[0][0] : part[0][2], send1 = b1 ? part[0][1] : part[0][3];
+      const float keep0 = b1 ? red[0][2] : red[0][0], keep1 = b1 ? red[0][3] : red[0][1];
+      const float send0 = b1 ? red[0][0] : red[0][2], send1 = b1 ? red[0][1] : red[0][3];
       const float r0 = keep0 + __shfl_xor_sync(kFull, send0, 2);
       const float r1 = keep1 + __shfl_xor_sync(kFull, send1, 2);
       float s_log = (b0 ? r1 : r0) + __shfl_xor_sync(kFull, b0 ? r0 : r1, 1);
@@ -284,29 +316,42 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
       psum += __shfl_xor_sync(kFull, psum, 16);
       l_run = fmaf(l_run, cr, psum);
       m_run = m_new;
-      prob[lane] = pw;
-      if (tok == 0) corr[hd] = cr;
+      prob[lane] = make_float2(pw, pw);
+      const bool rescale = __any_sync(kFull, cr != 1.f);   // the running maximum moved for some head
+      if (rescale && tok == 0) corr[hd] = make_float2(cr, cr);
       __syncwarp();
 
       // ---- P.V on this lane's channels -----------------------------------------------------------
-      const float4 c4 = *reinterpret_cast<const float4*>(corr);
-      const float cv[4] = {c4.x, c4.y, c4.z, c4.w};
+      if (rescale) {
+        const float4 c01 = *reinterpret_cast<const float4*>(corr);
+        const float4 c23 = *reinterpret_cast<const float4*>(corr + 2);
+        const float2 cv[4] = {make_float2(c01.x, c01.y), make_float2(c01.z, c01.w), make_float2(c23.x, c23.y),
+                              make_float2(c23.z, c23.w)};
 #pragma unroll
-      for (int hh = 0; hh < RH; ++hh)
+        for (int hh = 0; hh < RH; ++hh)
 #pragma unroll
-        for (int j = 0; j < DPL; ++j) acc[hh][j] *= cv[hh];
+          for (int j = 0; j < DPL / 2; ++j) acc[hh][j] = __fmul2_rn(acc[hh][j], cv[hh]);
+      }
+      auto pv_token = [&](int t) {
+        float vf[DPL];
+        lds_row<KV_T, DPL>(vbase + uint32_t(t) * ROWB, vf);
+        const float4 p01 = *reinterpret_cast<const float4*>(prob + 4 * t);
+        const float4 p23 = *reinterpret_cast<const float4*>(prob + 4 * t + 2);
+        const float2 pv[4] = {make_float2(p01.x, p01.y), make_float2(p01.z, p01.w), make_float2(p23.x, p23.y),
+                              make_float2(p23.z, p23.w)};
 #pragma unroll
-      for (int t = 0; t < kTok; ++t) {
-        if ((mask >> t) & 1u) {                     // warp-uniform; stale rows are never read
-          float vf[DPL];
-          lds_row<KV_T, DPL>(vbase + uint32_t(t) * ROWB, vf);
-          const float4 p4 = *reinterpret_cast<const float4*>(prob + 4 * t);
-          const float pv[4] = {p4.x, p4.y, p4.z, p4.w};
+        for (int hh = 0; hh < RH; ++hh)
 #pragma unroll
-          for (int hh = 0; hh < RH; ++hh)
+          for (int j = 0; j < DPL / 2; ++j)
+            acc[hh][j] = __ffma2_rn(pv[hh], make_float2(vf[2 * j], vf[2 * j + 1]), acc[hh][j]);
+      };
+      if (mask == (1u << kTok) - 1u) {
 #pragma unroll
-            for (int j = 0; j < DPL; ++j) acc[hh][j] = fmaf(pv[hh], vf[j], acc[hh][j]);
-        }
+        for (int t = 0; t < kTok; ++t) pv_token(t);
+      } else {
+#pragma unroll
+        for (int t = 0; t < kTok; ++t)
+          if ((mask >> t) & 1u) pv_token(t);          // warp-uniform; stale rows are never read
       }
     }
     __syncwarp();                                   // all lanes are done with the stage and prob[]
@@ -334,7 +379,8 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
 #pragma unroll
   for (int hh = 0; hh < RH; ++hh)
 #pragma unroll
-    for (int j = 0; j < DPL; ++j) sm_acc[(warp * RH + hh) * D + lane * DPL + j] = acc[hh][j];
+    for (int j = 0; j < DPL / 2; ++j)
+      *reinterpret_cast<float2*>(&sm_acc[(warp * RH + hh) * D + lane * DPL + 2 * j]) = acc[hh][j];
   __syncthreads();
   for (int i = threadIdx.x; i < RH * D; i += kThreads) {
     const int hh = i / D, c = i % D;
