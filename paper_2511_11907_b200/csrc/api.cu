@@ -125,7 +125,7 @@ int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* p
   float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
 
   cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
-  if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, stream);
+  if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
   if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }

@@ -48,7 +48,7 @@ cudaError_t launch_project_keys(const Problem& p, const void* K, const float* pr
 cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* proj, float* uq,
                                  cudaStream_t st);
 cudaError_t launch_score_pool(const Problem& p, const float* uq, const void* meta, float* scores,
-                              cudaStream_t st);
+                              uint32_t* err, cudaStream_t st);
 cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* group_idx,
                                int32_t* n_selected, cudaStream_t st);
 cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K,

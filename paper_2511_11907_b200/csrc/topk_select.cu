@@ -2,8 +2,14 @@
 // the largest score, lower index first among equal scores, written in ascending index order.
 //
 // One CTA per problem.  Scores become order-preserving 32-bit keys; an MSB-first radix select
-// (8 bits per pass) finds the key of rank M' and how many groups equal to it are still needed;
-// a stable compaction in index order then emits the selection.
+// finds the key of rank M' and how many groups equal to it are still needed; a stable compaction
+// in index order then emits the selection.
+//   topk_select_regs_kernel   NG <= 16384: every thread keeps its 1, 4 or 16 consecutive keys in
+//                             registers; digits of 12, 12 and 8 bits, so that the first pass
+//                             already isolates a few hundred candidates and later passes touch
+//                             only those; stops as soon as a digit bin is taken whole.
+//   topk_select_kernel        longer rows: keys in shared memory (or re-read), 8-bit digits.
+#include "async_copy.cuh"
 #include "common.cuh"
 
 namespace kvswap {
@@ -51,6 +57,8 @@ topk_select_kernel(Problem p, const float* __restrict__ scores, int32_t* __restr
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_want;
 
+  pdl_wait();
+  pdl_trigger();
   const int prob = blockIdx.x;                 // b * S + s
   const float* R = scores + int64_t(prob) * p.NG;
   int32_t* out = group_idx + int64_t(prob) * p.M;
@@ -115,18 +123,159 @@ topk_select_kernel(Problem p, const float* __restrict__ scores, int32_t* __restr
   }
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Register-resident select for NG <= kThreads * KPT.
+// ------------------------------------------------------------------------------------------
+constexpr int kBins = 4096;
+
+// Among the candidates counted in hist[0..n_bins) find, from the top, the bin that holds the
+// candidate of descending rank `want` (1-based).  Thread t owns `per` consecutive bins counted
+// down from the top.  Results: sh_bin, sh_want (rank inside that bin), sh_cnt (its population).
+__device__ __forceinline__ void find_bin(const int* hist, int n_bins, int want, int* warp_tot, int* sh_bin,
+                                         int* sh_want, int* sh_cnt) {
+  const int per = (n_bins + kThreads - 1) / kThreads;          // 4 for 4096 bins, 1 for 256
+  const int top = n_bins - 1 - int(threadIdx.x) * per;         // highest bin of this thread
+  int local = 0;
+  for (int i = 0; i < per; ++i) { const int bin = top - i; if (bin >= 0) local += hist[bin]; }
+  const int incl = block_inclusive_scan(local, warp_tot);
+  const int before = incl - local;                             // candidates in bins above mine
+  if (before < want && incl >= want) {
+    int acc = before;
+    for (int i = 0; i < per; ++i) {
+      const int bin = top - i;
+      const int c = (bin >= 0) ? hist[bin] : 0;
+      if (acc + c >= want) { *sh_bin = bin; *sh_want = want - acc; *sh_cnt = c; break; }
+      acc += c;
+    }
+  }
+}
+
+template <int KPT>
+__global__ void __launch_bounds__(kThreads)
+topk_select_regs_kernel(Problem p, const float* __restrict__ scores, int32_t* __restrict__ group_idx,
+                        int32_t* __restrict__ n_selected) {
+  __shared__ int hist[kBins];
+  __shared__ int warp_tot[32];
+  __shared__ int sh_bin, sh_want, sh_cnt;
+
+  const int prob = blockIdx.x;                 // b * S + s
+  const int NG = p.NG, Mp = p.Mp;
+  for (int i = threadIdx.x; i < kBins; i += kThreads) hist[i] = 0;
+  pdl_wait();
+  pdl_trigger();
+  const float* R = scores + int64_t(prob) * NG;
+  int32_t* out = group_idx + int64_t(prob) * p.M;
+
+  if (threadIdx.x == 0) n_selected[prob] = Mp;
+  for (int i = Mp + threadIdx.x; i < p.M; i += kThreads) out[i] = -1;
+  if (Mp == 0) return;
+  if (Mp == NG) {                              // everything is selected
+    for (int i = threadIdx.x; i < NG; i += kThreads) out[i] = i;
+    return;
+  }
+
+  // ---- this thread's KPT consecutive keys (0 = below every real key, for the padding) ----------
+  const int i0 = int(threadIdx.x) * KPT;
+  uint32_t key[KPT];
+  if constexpr (KPT >= 4) {
+    if ((NG & 3) == 0) {
+#pragma unroll
+      for (int v = 0; v < KPT / 4; ++v) {
+        if (i0 + 4 * v < NG) {
+          const float4 f = *reinterpret_cast<const float4*>(R + i0 + 4 * v);
+          key[4 * v] = score_key(f.x); key[4 * v + 1] = score_key(f.y);
+          key[4 * v + 2] = score_key(f.z); key[4 * v + 3] = score_key(f.w);
+        } else {
+          key[4 * v] = key[4 * v + 1] = key[4 * v + 2] = key[4 * v + 3] = 0u;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < KPT; ++e) key[e] = (i0 + e < NG) ? score_key(R[i0 + e]) : 0u;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < KPT; ++e) key[e] = (i0 + e < NG) ? score_key(R[i0 + e]) : 0u;
+  }
+  // A real key is never 0: score_key maps -NaN (all ones) to 0 only for the pattern 0xffffffff;
+  // give that one pattern the next key up so that padding stays strictly below every real key.
+#pragma unroll
+  for (int e = 0; e < KPT; ++e) if (i0 + e < NG && key[e] == 0u) key[e] = 1u;
+  __syncthreads();                             // hist is cleared
+
+  // ---- pass 1: top 12 bits of every key -----------------------------------------------------------
+#pragma unroll
+  for (int e = 0; e < KPT; ++e) if (i0 + e < NG) atomicAdd(&hist[key[e] >> 20], 1);
+  __syncthreads();
+  find_bin(hist, kBins, Mp, warp_tot, &sh_bin, &sh_want, &sh_cnt);
+  __syncthreads();
+  uint32_t prefix = uint32_t(sh_bin) << 20;    // known high bits of the M'-th key
+  uint32_t known = 0xfff00000u;
+  int want = sh_want, cnt = sh_cnt;
+  uint32_t kth;                                // keys > kth are selected, plus need_eq keys == kth
+  int need_eq;
+  if (cnt == want) { kth = prefix - 1u; need_eq = 0; }        // the whole bin is taken (prefix > 0 here)
+  else {
+    // ---- pass 2: next 12 bits of the candidates ------------------------------------------------------
+    for (int i = threadIdx.x; i < kBins; i += kThreads) hist[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < KPT; ++e)
+      if ((key[e] & known) == prefix && i0 + e < NG) atomicAdd(&hist[(key[e] >> 8) & 0xfffu], 1);
+    __syncthreads();
+    find_bin(hist, kBins, want, warp_tot, &sh_bin, &sh_want, &sh_cnt);
+    __syncthreads();
+    prefix |= uint32_t(sh_bin) << 8;
+    known = 0xffffff00u;
+    want = sh_want; cnt = sh_cnt;
+    if (cnt == want) { kth = prefix - 1u; need_eq = 0; }
+    else {
+      // ---- pass 3: last 8 bits ---------------------------------------------------------------------
+      if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+      __syncthreads();
+#pragma unroll
+      for (int e = 0; e < KPT; ++e)
+        if ((key[e] & known) == prefix && i0 + e < NG) atomicAdd(&hist[key[e] & 0xffu], 1);
+      __syncthreads();
+      find_bin(hist, 256, want, warp_tot, &sh_bin, &sh_want, &sh_cnt);
+      __syncthreads();
+      kth = prefix | uint32_t(sh_bin);
+      need_eq = sh_want;                       // equal keys to take, lowest indices first
+    }
+  }
+
+  // ---- stable compaction in index order: one scan carries both counts ----------------------------------
+  int n_gt = 0, n_eq = 0;
+#pragma unroll
+  for (int e = 0; e < KPT; ++e) { n_gt += (key[e] > kth); n_eq += (key[e] == kth); }
+  const int packed = block_inclusive_scan((n_gt << 16) | n_eq, warp_tot) - ((n_gt << 16) | n_eq);
+  const int gt_before = packed >> 16, eq_before = packed & 0xffff;
+  int eq_take = max(0, min(n_eq, need_eq - eq_before));
+  int pos = gt_before + min(eq_before, need_eq);
+#pragma unroll
+  for (int e = 0; e < KPT; ++e) {
+    bool take = key[e] > kth;
+    if (key[e] == kth && eq_take > 0) { take = true; --eq_take; }
+    if (take) out[pos++] = i0 + e;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* group_idx, int32_t* n_selected,
                                cudaStream_t st) {
+  const dim3 grid(p.B * p.S), block(kThreads);
+  if (p.NG <= kThreads) return launch_pdl(topk_select_regs_kernel<1>, grid, block, 0, st, p, scores, group_idx, n_selected);
+  if (p.NG <= 4 * kThreads) return launch_pdl(topk_select_regs_kernel<4>, grid, block, 0, st, p, scores, group_idx, n_selected);
+  if (p.NG <= 16 * kThreads) return launch_pdl(topk_select_regs_kernel<16>, grid, block, 0, st, p, scores, group_idx, n_selected);
   const int keys_in_smem = (p.NG <= kMaxSmemKeys) ? 1 : 0;
   const size_t smem = keys_in_smem ? sizeof(uint32_t) * size_t(p.NG) : 0;
   if (smem > 40 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
   }
-  topk_select_kernel<<<p.B * p.S, kThreads, smem, st>>>(p, scores, group_idx, n_selected, keys_in_smem);
-  return cudaGetLastError();
+  return launch_pdl(topk_select_kernel, grid, block, smem, st, p, scores, group_idx, n_selected, keys_in_smem);
 }
 
 }  // namespace kvswap
