@@ -110,6 +110,7 @@ constexpr int kRowBytes = 64;
 constexpr int kTileBytes = kTileRows * kRowBytes;
 constexpr int kWarps = 8;
 constexpr int kDepth = 4;
+constexpr int kOutStride = kTileRows + 1;   // padded row of the per-warp output tile (bank spread)
 
 struct TileControl {
   unsigned long long full[kWarps * kDepth];
@@ -139,7 +140,7 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
   extern __shared__ __align__(128) unsigned char dyn[];
   unsigned char* tiles = dyn;                                                       // [kWarps][kDepth][kTileBytes]
   TileControl* ctl = reinterpret_cast<TileControl*>(dyn + kWarps * kDepth * kTileBytes);
-  float* outbuf = reinterpret_cast<float*>(dyn + kWarps * kDepth * kTileBytes + sizeof(TileControl));  // [kWarps][NS][kTileRows]
+  float* outbuf = reinterpret_cast<float*>(dyn + kWarps * kDepth * kTileBytes + sizeof(TileControl));  // [kWarps][NS][kOutStride]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rq = lane >> 2, qt = lane & 3;          // row within a read, quarter of the row
@@ -162,13 +163,17 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
   int c_tile = f_tile, c_rest = f_rest;                                   // next item to consume
 
   const uint32_t ring = smem_addr(tiles) + uint32_t(warp) * kDepth * kTileBytes;
+  const META_T* f_base = nullptr;                   // metadata of the fill cursor's (sequence, head)
+  int f_base_rest = -1;
   auto fill = [&](int stage) {                      // requests the item under the fill cursor
     if (lane == 0) {
-      const int bh = f_rest / n_sub;
-      const int hm = bh % hm_count, b = bh / hm_count;
+      if (f_rest != f_base_rest) {
+        f_base_rest = f_rest;
+        const int bh = f_rest / n_sub;
+        f_base = meta + int64_t(bh / hm_count) * p.meta_sb + int64_t(bh % hm_count) * p.meta_sh;
+      }
       const int rows = min(kTileRows, rows_total - f_tile * kTileRows);
-      const META_T* src = meta + int64_t(b) * p.meta_sb + int64_t(hm) * p.meta_sh +
-                          int64_t(f_tile) * kTileRows * p.meta_sn;
+      const META_T* src = f_base + int64_t(f_tile) * kTileRows * p.meta_sn;
       const uint32_t bar = smem_addr(&ctl->full[warp * kDepth + stage]);
       mbar_arrive_expect_tx(bar, uint32_t(rows) * kRowBytes);
       bulk_g2s(ring + uint32_t(stage) * kTileBytes, src, uint32_t(rows) * kRowBytes, bar);
@@ -192,7 +197,7 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
 #pragma unroll
   for (int i = 0; i < NV; ++i) vmax[i] = -INFINITY;
   const int gb = (g_shift < 3) ? g_shift : 3;       // butterfly levels over the row bits
-  float* out = outbuf + warp * (NS * kTileRows);
+  float* out = outbuf + warp * (NS * kOutStride);
   int stage = 0;
   uint32_t phase = 0;
   bool timed_out = false;
@@ -224,10 +229,11 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
       float v[NS];
 #pragma unroll
       for (int c = 0; c < NS; ++c) {
-        float2 a = __fmul2_rn(uu[c][0], m[0]);
+        float a = uu[c][0].x * m[0].x;
+        a = fmaf(uu[c][0].y, m[0].y, a);
 #pragma unroll
-        for (int i = 1; i < KP; ++i) a = __ffma2_rn(uu[c][i], m[i], a);
-        v[c] = a.x + a.y;
+        for (int i = 1; i < KP; ++i) { a = fmaf(uu[c][i].x, m[i].x, a); a = fmaf(uu[c][i].y, m[i].y, a); }
+        v[c] = a;
       }
       // ---- the four lanes of a row: reduce-scatter of the NS partial scores -----------------
       if constexpr (NS >= 8) {
@@ -261,7 +267,7 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
         const int gi = (it * 8 + rq) >> g_shift;    // group within the tile
         if ((rq & ((1 << gb) - 1)) == 0) {
 #pragma unroll
-          for (int i = 0; i < NV; ++i) out[((i ^ perm) & (NS - 1)) * kTileRows + gi] = vmax[i];
+          for (int i = 0; i < NV; ++i) out[((i ^ perm) & (NS - 1)) * kOutStride + gi] = vmax[i];
         }
 #pragma unroll
         for (int i = 0; i < NV; ++i) vmax[i] = -INFINITY;
@@ -276,7 +282,7 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
       const int ns = (p.Hm == 1) ? min(NS, p.S - s0) : 1;
       for (int i = lane; i < ns * ngt; i += 32) {
         const int s = i / ngt, gi = i - s * ngt;
-        scores[(int64_t(b) * p.S + s0 + s) * p.NG + g0 + gi] = out[s * kTileRows + gi];
+        scores[(int64_t(b) * p.S + s0 + s) * p.NG + g0 + gi] = out[s * kOutStride + gi];
       }
     }
     __syncwarp();                                   // stage and outbuf are free again
@@ -286,6 +292,198 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
   if (timed_out) {
     if (lane == 0 && err) atomicExch(err, kDevTimeoutFull);
     for (int s = 0; s < kDepth; ++s) {              // bounded chance for copies in flight to land
+      mbar_wait(smem_addr(&ctl->full[warp * kDepth + s]), 0);
+      mbar_wait(smem_addr(&ctl->full[warp * kDepth + s]), 1);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// K2, streaming path for joint fp16 metadata scored for several scopes at once.
+//
+// With one metadata row feeding up to 8 scores (the per-KV-head scopes of the joint adapter) the
+// work per row is an [rows x 32] . [32 x 8] contraction at 8 FLOP per byte, which the fp32 pipes
+// cannot sustain at HBM rate; it runs on the tensor cores instead (mma.sync m16n8k16, fp16 inputs,
+// fp32 accumulation), 16 rows per instruction group.  The summed low-rank queries stay fp32-exact:
+// each is scaled by a power of two and split into an fp16 head and an fp16 remainder (two
+// products per k-step), so the only rounding is the accumulator's.
+//
+// Operand layout.  A 16-byte shared-memory read gives lane (g = lane / 4, t = lane % 4) the rank
+// entries 8t..8t+7 of row g.  The contraction index may be permuted freely as long as both
+// operands agree, so k-step j takes entries 8t+4j..8t+4j+3 as the four A values the lane owes for
+// its row, and the lane's B values are the same entries of the query of scope g.  The
+// accumulator then holds rows g and g+8 for scopes 2t and 2t+1.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_half2(__half lo, __half hi) {
+  return uint32_t(__half_as_ushort(lo)) | (uint32_t(__half_as_ushort(hi)) << 16);
+}
+
+__global__ void __launch_bounds__(kWarps * 32, 2)
+score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __restrict__ meta,
+                      float* __restrict__ scores, int tiles_per_row, int n_sub, int g_shift,
+                      uint32_t* __restrict__ err) {
+  constexpr int NS = 8;
+  extern __shared__ __align__(128) unsigned char dyn[];
+  unsigned char* tiles = dyn;
+  TileControl* ctl = reinterpret_cast<TileControl*>(dyn + kWarps * kDepth * kTileBytes);
+  float* outbuf = reinterpret_cast<float*>(dyn + kWarps * kDepth * kTileBytes + sizeof(TileControl));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rq = lane >> 2, qt = lane & 3;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kWarps * kDepth; ++s) mbar_init(smem_addr(&ctl->full[s]), 1);
+    mbar_init_fence();
+  }
+  __syncthreads();
+
+  const int rows_total = p.NG * p.G;
+  const int64_t items = int64_t(p.B) * n_sub * tiles_per_row;
+  const int64_t gw = int64_t(blockIdx.x) * kWarps + warp, n_gw = int64_t(gridDim.x) * kWarps;
+  const int first = int(items * gw / n_gw), last = int(items * (gw + 1) / n_gw);
+  const int my_tiles = last - first;
+  int f_tile = first % tiles_per_row, f_rest = first / tiles_per_row;     // rest = b * n_sub + sub
+  int c_tile = f_tile, c_rest = f_rest;
+
+  const uint32_t ring = smem_addr(tiles) + uint32_t(warp) * kDepth * kTileBytes;
+  auto fill = [&](int stage) {
+    if (lane == 0) {
+      const int rows = min(kTileRows, rows_total - f_tile * kTileRows);
+      const __half* src = meta + int64_t(f_rest / n_sub) * p.meta_sb + int64_t(f_tile) * kTileRows * p.meta_sn;
+      const uint32_t bar = smem_addr(&ctl->full[warp * kDepth + stage]);
+      mbar_arrive_expect_tx(bar, uint32_t(rows) * kRowBytes);
+      bulk_g2s(ring + uint32_t(stage) * kTileBytes, src, uint32_t(rows) * kRowBytes, bar);
+    }
+    if (++f_tile == tiles_per_row) { f_tile = 0; ++f_rest; }
+  };
+  // The metadata is never written by the kernel that precedes this one in the same call.
+  for (int k = 0; k < kDepth && k < my_tiles; ++k) fill(k);
+  pdl_wait();
+  pdl_trigger();
+
+  uint32_t bhi[2][2], blo[2][2];                    // B fragments of k-steps 0 and 1
+  float inv0 = 1.f, inv1 = 1.f;                     // undo the scaling of scopes 2t and 2t+1
+  int cur_rest = -1, b = 0, sub = 0;
+  const int gb = (g_shift < 3) ? g_shift : 3;
+  float run0 = -INFINITY, run1 = -INFINITY;         // running maxima of a 32-row group
+  float* out = outbuf + warp * (NS * kOutStride);
+  int stage = 0;
+  uint32_t phase = 0;
+  bool timed_out = false;
+  for (int k = 0; k < my_tiles; ++k) {
+    const int tile = c_tile;
+    if (c_rest != cur_rest) {                       // new (sequence, scope block): rebuild B
+      cur_rest = c_rest;
+      sub = c_rest % n_sub; b = c_rest / n_sub;
+      const int sc = sub * NS + rq;                 // this lane supplies the query of scope sc
+      float u[8];
+      if (sc < p.S) {
+        const float4* ur = reinterpret_cast<const float4*>(uq + (int64_t(b) * p.Su + sc) * p.r + qt * 8);
+        const float4 x = ur[0], y = ur[1];
+        u[0] = x.x; u[1] = x.y; u[2] = x.z; u[3] = x.w; u[4] = y.x; u[5] = y.y; u[6] = y.z; u[7] = y.w;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) u[i] = 0.f;
+      }
+      float mx = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fabsf(u[i]));
+      mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+      // power of two that brings the largest entry into [2^14, 2^15)
+      int sh = 0;
+      if (mx > 0.f && mx < INFINITY) sh = min(120, max(-113, 14 - (int((__float_as_uint(mx) >> 23) & 0xffu) - 127)));
+      const float scale = __uint_as_float(uint32_t(sh + 127) << 23);
+      const float inv = __uint_as_float(uint32_t(127 - sh) << 23);
+      __half hi[8], lo[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float us = u[i] * scale;
+        hi[i] = __float2half_rn(us);
+        lo[i] = __float2half_rn(us - __half2float(hi[i]));
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        bhi[j][0] = pack_half2(hi[4 * j], hi[4 * j + 1]); bhi[j][1] = pack_half2(hi[4 * j + 2], hi[4 * j + 3]);
+        blo[j][0] = pack_half2(lo[4 * j], lo[4 * j + 1]); blo[j][1] = pack_half2(lo[4 * j + 2], lo[4 * j + 3]);
+      }
+      inv0 = __shfl_sync(kFull, inv, (2 * qt) * 4);
+      inv1 = __shfl_sync(kFull, inv, (2 * qt + 1) * 4);
+    }
+    if (++c_tile == tiles_per_row) { c_tile = 0; ++c_rest; }
+    if (!__all_sync(kFull, mbar_wait(smem_addr(&ctl->full[warp * kDepth + stage]), phase))) { timed_out = true; break; }
+    const int rows = min(kTileRows, rows_total - tile * kTileRows);
+    const int ngt = rows >> g_shift;                // groups in this tile
+    const uint32_t base = ring + uint32_t(stage) * kTileBytes + uint32_t(lane) * 16u;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      if (mt * 16 < rows) {
+        uint32_t wa[4], wb[4];                      // rows g and g + 8 of this 16-row block
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(wa[0]), "=r"(wa[1]), "=r"(wa[2]), "=r"(wa[3])
+                     : "r"(base + uint32_t(mt) * 16u * kRowBytes));
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(wb[0]), "=r"(wb[1]), "=r"(wb[2]), "=r"(wb[3])
+                     : "r"(base + uint32_t(mt) * 16u * kRowBytes + 8u * kRowBytes));
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          mma16816(d, wa[2 * j], wb[2 * j], wa[2 * j + 1], wb[2 * j + 1], bhi[j][0], bhi[j][1]);
+          mma16816(d, wa[2 * j], wb[2 * j], wa[2 * j + 1], wb[2 * j + 1], blo[j][0], blo[j][1]);
+        }
+        float x0 = d[0] * inv0, x1 = d[1] * inv1;   // row g,     scopes 2t, 2t+1
+        float y0 = d[2] * inv0, y1 = d[3] * inv1;   // row g + 8, scopes 2t, 2t+1
+        if (g_shift >= 4) { x0 = fmaxf(x0, y0); x1 = fmaxf(x1, y1); }
+        if (gb >= 1) {
+          x0 = fmaxf(x0, __shfl_xor_sync(kFull, x0, 4)); x1 = fmaxf(x1, __shfl_xor_sync(kFull, x1, 4));
+          y0 = fmaxf(y0, __shfl_xor_sync(kFull, y0, 4)); y1 = fmaxf(y1, __shfl_xor_sync(kFull, y1, 4));
+        }
+        if (gb >= 2) {
+          x0 = fmaxf(x0, __shfl_xor_sync(kFull, x0, 8)); x1 = fmaxf(x1, __shfl_xor_sync(kFull, x1, 8));
+          y0 = fmaxf(y0, __shfl_xor_sync(kFull, y0, 8)); y1 = fmaxf(y1, __shfl_xor_sync(kFull, y1, 8));
+        }
+        if (gb >= 3) {
+          x0 = fmaxf(x0, __shfl_xor_sync(kFull, x0, 16)); x1 = fmaxf(x1, __shfl_xor_sync(kFull, x1, 16));
+          y0 = fmaxf(y0, __shfl_xor_sync(kFull, y0, 16)); y1 = fmaxf(y1, __shfl_xor_sync(kFull, y1, 16));
+        }
+        if ((rq & ((1 << gb) - 1)) == 0) {          // lanes of a group's first row publish it
+          float* o0 = out + (2 * qt) * kOutStride;
+          float* o1 = o0 + kOutStride;
+          if (g_shift <= 3) {
+            const int gx = (mt * 16 + rq) >> g_shift, gy = (mt * 16 + 8 + rq) >> g_shift;
+            if (gx < ngt) { o0[gx] = x0; o1[gx] = x1; }
+            if (gy < ngt) { o0[gy] = y0; o1[gy] = y1; }
+          } else if (g_shift == 4) {
+            o0[mt] = x0; o1[mt] = x1;
+          } else {                                  // G = 32: the tile is one group
+            run0 = fmaxf(run0, x0); run1 = fmaxf(run1, x1);
+            if (mt == 1) { o0[0] = run0; o1[0] = run1; run0 = -INFINITY; run1 = -INFINITY; }
+          }
+        }
+      }
+    }
+    __syncwarp();
+    {
+      const int g0 = (tile * kTileRows) >> g_shift;
+      const int s0 = sub * NS;
+      const int ns = min(NS, p.S - s0);
+      for (int i = lane; i < ns * ngt; i += 32) {
+        const int s = i / ngt, gi = i - s * ngt;
+        scores[(int64_t(b) * p.S + s0 + s) * p.NG + g0 + gi] = out[s * kOutStride + gi];
+      }
+    }
+    __syncwarp();
+    if (k + kDepth < my_tiles) fill(stage);
+    if (++stage == kDepth) { stage = 0; phase ^= 1u; }
+  }
+  if (timed_out) {
+    if (lane == 0 && err) atomicExch(err, kDevTimeoutFull);
+    for (int s = 0; s < kDepth; ++s) {
       mbar_wait(smem_addr(&ctl->full[warp * kDepth + s]), 0);
       mbar_wait(smem_addr(&ctl->full[warp * kDepth + s]), 1);
     }
@@ -398,12 +596,28 @@ cudaError_t launch_tiles(const Problem& p, const float* uq, const void* meta, fl
   // One wave of two CTAs per SM; fewer CTAs when there is not at least one tile per warp.
   const int64_t want = (items + kWarps - 1) / kWarps;
   const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(2 * kNumSMs, want)));
-  const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kTileRows;
+  const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kOutStride;
   auto kern = score_pool_tiles_kernel<META_T, NS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
   if (e != cudaSuccess) return e;
   return launch_pdl(kern, dim3(ctas), dim3(kWarps * 32), smem, st, p, uq, static_cast<const META_T*>(meta), scores,
                     tiles_per_row, n_sub, g_shift, err);
+}
+
+cudaError_t launch_mma(const Problem& p, const float* uq, const void* meta, float* scores, int g_shift,
+                       uint32_t* err, cudaStream_t st) {
+  constexpr int NS = 8;
+  const int rows_total = p.NG * p.G;
+  const int tiles_per_row = (rows_total + kTileRows - 1) / kTileRows;
+  const int n_sub = (p.S + NS - 1) / NS;
+  const int64_t items = int64_t(p.B) * n_sub * tiles_per_row;
+  const int64_t want = (items + kWarps - 1) / kWarps;
+  const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(2 * kNumSMs, want)));
+  const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kOutStride;
+  cudaError_t e = cudaFuncSetAttribute(score_pool_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+  if (e != cudaSuccess) return e;
+  return launch_pdl(score_pool_mma_kernel, dim3(ctas), dim3(kWarps * 32), smem, st, p, uq,
+                    static_cast<const __half*>(meta), scores, tiles_per_row, n_sub, g_shift, err);
 }
 
 template <typename META_T>
@@ -417,6 +631,9 @@ cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, flo
                          tile_items < (int64_t(1) << 30);
   if (streaming) {
     const int ns = (p.Hm == 1) ? p.S : 1;
+    if constexpr (std::is_same<META_T, __half>::value) {
+      if (ns >= 3) return launch_mma(p, uq, meta, scores, g_shift, err, st);
+    }
     if (ns == 1) return launch_tiles<META_T, 1>(p, uq, meta, scores, g_shift, err, st);
     if (ns == 2) return launch_tiles<META_T, 2>(p, uq, meta, scores, g_shift, err, st);
     if (ns <= 4) return launch_tiles<META_T, 4>(p, uq, meta, scores, g_shift, err, st);
