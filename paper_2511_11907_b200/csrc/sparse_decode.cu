@@ -402,27 +402,51 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   }
 }
 
-// K5: merge the split partials of one (sequence, head).
+// K5: merge the split partials of one (sequence, head).  One CTA of D threads per row; every
+// load of the row is issued before anything is computed (one memory round trip), the split
+// weights are formed once by the first warp and shared.
+constexpr int kMaxSplits = 256;
+
 template <int D>
 __global__ void __launch_bounds__(D)
 combine_kernel(const float* __restrict__ partial, float* __restrict__ out, float* __restrict__ lse, int splits) {
+  __shared__ float w_s[kMaxSplits];
+  __shared__ float norm_s[2];                  // 1 / sum of weights (or 0), lse
   pdl_wait();
   pdl_trigger();
   const int64_t bh = blockIdx.x;
   const float* src = partial + bh * splits * (D + 2);
   const int c = threadIdx.x;
-  float mx = -INFINITY;
-  for (int s = 0; s < splits; ++s) mx = fmaxf(mx, src[s * (D + 2)]);
-  float lsum = 0.f, a = 0.f;
-  if (mx > -INFINITY) {
-    for (int s = 0; s < splits; ++s) {
-      const float w = exp2f(src[s * (D + 2)] - mx);
+  constexpr int kUnroll = 16;
+  float a_first[kUnroll];
+#pragma unroll
+  for (int s = 0; s < kUnroll; ++s) a_first[s] = (s < splits) ? src[s * (D + 2) + 2 + c] : 0.f;
+  if (c < 32) {
+    // weights: lane s handles splits s, s + 32, ...
+    float mx = -INFINITY;
+    for (int s = c; s < splits; s += 32) mx = fmaxf(mx, src[s * (D + 2)]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    float lsum = 0.f;
+    for (int s = c; s < splits; s += 32) {
+      const float w = (mx > -INFINITY) ? exp2f(src[s * (D + 2)] - mx) : 0.f;
+      w_s[s] = w;
       lsum = fmaf(src[s * (D + 2) + 1], w, lsum);
-      a = fmaf(src[s * (D + 2) + 2 + c], w, a);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, off);
+    if (c == 0) {
+      norm_s[0] = (lsum > 0.f) ? 1.f / lsum : 0.f;
+      norm_s[1] = (lsum > 0.f) ? (mx + log2f(lsum)) * kLn2 : -INFINITY;
     }
   }
-  out[bh * D + c] = (lsum > 0.f) ? a / lsum : 0.f;
-  if (lse != nullptr && c == 0) lse[bh] = (lsum > 0.f) ? (mx + log2f(lsum)) * kLn2 : -INFINITY;
+  __syncthreads();
+  float a = 0.f;
+#pragma unroll
+  for (int s = 0; s < kUnroll; ++s) if (s < splits) a = fmaf(a_first[s], w_s[s], a);
+  for (int s = kUnroll; s < splits; ++s) a = fmaf(src[s * (D + 2) + 2 + c], w_s[s], a);
+  out[bh * D + c] = a * norm_s[0];
+  if (lse != nullptr && c == 0) lse[bh] = norm_s[1];
 }
 
 template <typename KV_T, int D>
