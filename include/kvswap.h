@@ -69,7 +69,7 @@ typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_sco
  *   meta_* strides (in elements) of the metadata, laid out [B, H_m, N, r].
  * A stride of 0 means "dense": the natural stride of the contiguous tensor.
  * Supported ranges: d in {64, 128}; r a multiple of 4 with 4 <= r <= 256; G >= 1; M >= 1;
- * rho >= 1; G <= 1024; kv_dtype in {F32, BF16, F16}; q_dtype = kv_dtype or F32; meta_dtype in
+ * rho >= 1; G <= 1024; M * G <= 2^30; kv_dtype in {F32, BF16, F16}; q_dtype = kv_dtype or F32; meta_dtype in
  * {F32, F16}.
  */
 typedef struct {

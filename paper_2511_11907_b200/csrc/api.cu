@@ -32,6 +32,7 @@ int resolve(const kvswap_shape* s, Problem* p) {
   if (s->q_dtype != KVSWAP_F32 && s->q_dtype != s->kv_dtype) return KVSWAP_ERR_DTYPE;  // q: fp32 or K/V's type
   if (s->head_dim != 64 && s->head_dim != 128) return KVSWAP_ERR_UNSUPPORTED;
   if (s->rank % 4 != 0 || s->rank > 256 || s->group_size > 1024) return KVSWAP_ERR_UNSUPPORTED;
+  if (int64_t(s->top_k) * s->group_size > (int64_t(1) << 30)) return KVSWAP_ERR_UNSUPPORTED;
   if ((int64_t(s->rank) * em) % 16 != 0) return KVSWAP_ERR_ALIGN;
   if ((int64_t(s->head_dim) * eq) % 16 != 0) return KVSWAP_ERR_ALIGN;
 

@@ -3,8 +3,8 @@
 // log-sum-exp merge of the split partials.
 //
 // The attended tokens of one (sequence, selection row) form a virtual list
-//     v in [0, n_sel*G):  token  group_idx[v / G] * G + v % G
-//     v in [n_sel*G, n_sel*G + tail):  token  NG*G + (v - n_sel*G)
+//     v in [0, M*G):  token  group_idx[v / G] * G + v % G   (absent when v / G >= n_sel or the index is invalid)
+//     v in [M*G, M*G + tail):  token  NG*G + (v - M*G)
 // which is cut into `splits` contiguous ranges, one CTA each, and every range into chunks of
 // kTok tokens.  A CTA serves RH query heads that share the KV head, so each K/V row is read once.
 //
@@ -433,20 +433,22 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   pdl_wait();
   pdl_trigger();
 
+  // The virtual token list is laid out for M selected groups, whatever n_selected says (slots of
+  // groups beyond n_selected are simply absent), so that the split of the list does not wait for a
+  // global read: n_selected is fetched together with the first group indices.
   TokenSource src;
   src.idx = group_idx + (int64_t(b) * p.S + srow) * p.M;
   src.NG = p.NG; src.G = p.G; src.g_shift = g_shift;
+  src.tail0 = p.NG * p.G;
+  src.sel_tokens = p.M * p.G;
   {
-    int n_sel = n_selected[int64_t(b) * p.S + srow];
-    n_sel = max(0, min(n_sel, p.M));
-    src.tail0 = p.NG * p.G;
-    src.sel_tokens = n_sel * p.G;
     const int total = src.sel_tokens + (p.N - src.tail0);
     int per_split = (total + splits - 1) / splits;
     per_split = (per_split + kTok - 1) / kTok * kTok;
     src.v_begin = min(total, per_split * split);
     src.v_end = min(total, src.v_begin + per_split);
   }
+  const int n_sel = max(0, min(n_selected[int64_t(b) * p.S + srow], p.M));
   const int n_chunks = (src.v_end - src.v_begin + kTok - 1) / kTok;
   const int my_chunks = (n_chunks > warp) ? (n_chunks - warp + kWarps - 1) / kWarps : 0;   // of this warp
 
@@ -458,7 +460,10 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   // global read of the fill path, issued early so that its latency hides behind a chunk's compute.
   auto fetch_group = [&](int k) -> int {
     const int v = src.v_begin + (warp + k * kWarps) * kTok + lane;
-    if (lane < kTok && k < my_chunks && v < src.v_end && v < src.sel_tokens) return src.idx[src.group_of(v)];
+    if (lane < kTok && k < my_chunks && v < src.v_end && v < src.sel_tokens) {
+      const int go = src.group_of(v);
+      if (go < n_sel) return src.idx[go];
+    }
     return -1;
   };
   // Fill: bring chunk k into `stage` (one commit group).  `j` is fetch_group(k).  All lanes call.
@@ -662,7 +667,7 @@ void plan_sparse_decode(const Problem& p, Workspace* w) {
   for (int c = 4; c >= 1; --c) if (p.rho % c == 0) { rh = c; break; }
   w->heads_per_cta = rh;
   const int64_t problems = int64_t(p.B) * p.Hkv * (p.rho / rh);
-  const int64_t tokens = int64_t(p.Mp) * p.G + (p.N - int64_t(p.NG) * p.G);
+  const int64_t tokens = int64_t(p.M) * p.G + (p.N - int64_t(p.NG) * p.G);
   const int64_t n_chunks = std::max<int64_t>(1, (tokens + kTok - 1) / kTok);
   // One wave of 2 CTAs per SM when the problems are few; otherwise the split that fills whole
   // waves best, keeping at least two chunks per compute warp and split.
