@@ -1,8 +1,17 @@
-// K1: metadata build K_lr = Flatten(K) A (Sec. 4.2).
+// K1: metadata build K_lr = Flatten(K) A (Sec. 4.2) -- the dense contraction of the path.
 //
-// Generic shared-memory tiled contraction on the fp32 pipes: every (kv, meta) dtype pair, any
-// supported d and r.  A CTA owns 64 tokens x r outputs and walks the contraction index
-// (g, c) in chunks of 32 channels.
+//   project_keys_mma_kernel  bf16 K, r in {16, 32, 64}: tensor cores (mma.sync m16n8k16, fp32
+//                            accumulation).  The adapter stays fp32-exact: every entry is split
+//                            into three bf16 pieces (8 + 8 + 8 mantissa bits) and each k-step is
+//                            issued once per piece, so the products are exact and the only
+//                            rounding is the accumulator's and the final one into the metadata
+//                            type.  K rows go from global memory straight into A fragments; the
+//                            pre-split adapter of every KV head lives in shared memory as ready
+//                            B fragments for the whole kernel (persistent CTAs, one per SM).
+//   project_keys_kernel      every other case: shared-memory tiled contraction on the fp32
+//                            pipes (a CTA owns 64 tokens x r outputs, chunks of 32 channels).
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace kvswap {
@@ -91,6 +100,207 @@ project_keys_kernel(Problem p, const KV_T* __restrict__ K, const float* __restri
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Tensor-core path.
+//
+// Work item = (sequence b, metadata head hm, tile of 32 tokens); every warp of the grid takes an
+// equal contiguous share.  For an item a warp holds two 16-token accumulator tiles [16 x r] and
+// walks the contraction index head by head, 32 channels at a time: lane (g = lane / 4,
+// t = lane % 4) reads the 16 bytes of channels 32kk + 8t .. +7 of rows g and g + 8 of each tile.
+// The contraction index may be permuted as long as both operands agree, so those eight channels
+// serve as the lane's A values of two consecutive k-steps, and the B fragments in shared memory
+// are built with the same permutation.  The reads of the next half head are in flight while the
+// current one is multiplied.
+// ------------------------------------------------------------------------------------------
+constexpr int kMmaWarps = 12;
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <typename META_T, int D, int NT>            // NT = r / 8 output tiles of 8 columns
+__global__ void __launch_bounds__(kMmaWarps * 32, 1)
+project_keys_mma_kernel(Problem p, const __nv_bfloat16* __restrict__ K, const float* __restrict__ proj,
+                        META_T* __restrict__ meta, int n_begin, int n_end, int tiles_per_row) {
+  constexpr int KS = D / 16;                         // k-steps per head
+  constexpr int KK = D / 32;                         // 32-channel blocks per head
+  constexpr int HALF = (KK >= 2) ? 2 : 1;            // blocks multiplied per pipeline step
+  constexpr int STEPS_PER_HEAD = KK / HALF;
+  extern __shared__ __align__(16) unsigned char dyn[];
+  uint2* bfrag = reinterpret_cast<uint2*>(dyn);      // [H_kv][KS][NT][3 pieces][32 lanes]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g8 = lane >> 2, t4 = lane & 3;
+  const int r = NT * 8;
+
+  // ---- adapter -> B fragments, three bf16 pieces per entry ------------------------------------------
+  for (int i = threadIdx.x; i < p.Hkv * KS * NT * 32; i += kMmaWarps * 32) {
+    const int ln = i & 31, nt = (i >> 5) % NT, ks = ((i >> 5) / NT) % KS, g = (i >> 5) / (NT * KS);
+    const int t = ln & 3, col = nt * 8 + (ln >> 2);
+    const int c0 = 32 * (ks >> 1) + 8 * t + 4 * (ks & 1);      // channels c0 .. c0+3 feed this lane's k slots
+    const float* src = proj + (int64_t(g) * D + c0) * r + col;
+    float v[4], hi[4], mid[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      v[e] = src[int64_t(e) * r];
+      hi[e] = __bfloat162float(__float2bfloat16_rn(v[e]));
+      mid[e] = __bfloat162float(__float2bfloat16_rn(v[e] - hi[e]));
+      lo[e] = v[e] - hi[e] - mid[e];                 // exact; rounds to bf16 below
+    }
+    uint2* dst = bfrag + (int64_t(i >> 5) * 3) * 32 + ln;
+    dst[0] = make_uint2(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]));
+    dst[32] = make_uint2(pack_bf16(mid[0], mid[1]), pack_bf16(mid[2], mid[3]));
+    dst[64] = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
+  }
+  __syncthreads();
+
+  const int g_count = (p.Hm == 1) ? p.Hkv : 1;
+  const int64_t items = int64_t(p.B) * p.Hm * tiles_per_row;
+  const int64_t gw = int64_t(blockIdx.x) * kMmaWarps + warp, n_gw = int64_t(gridDim.x) * kMmaWarps;
+  const int64_t first = items * gw / n_gw, last = items * (gw + 1) / n_gw;
+
+  for (int64_t item = first; item < last; ++item) {
+    const int tile = int(item % tiles_per_row);
+    const int bh = int(item / tiles_per_row);
+    const int hm = bh % p.Hm, b = bh / p.Hm;
+    const int g_first = (p.Hm == 1) ? 0 : hm;
+    const int n0 = n_begin + tile * 32;
+    // rows of this lane: tile m, half h -> token n0 + 16 m + 8 h + g8
+    const __nv_bfloat16* rowp[2][2];
+    bool rowok[2][2];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int n = n0 + 16 * m + 8 * h + g8;
+        rowok[m][h] = n < n_end;
+        rowp[m][h] = K + int64_t(b) * p.kv_sb + int64_t(rowok[m][h] ? n : n_begin) * p.kv_sn + 8 * t4;
+      }
+    float acc[2][NT][4];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[m][nt][e] = 0.f;
+
+    auto load_step = [&](int step, uint4 (&a)[2][2][HALF]) {   // step = head-in-item * STEPS_PER_HEAD + half
+      const int g = g_first + step / STEPS_PER_HEAD;
+      const int kk0 = (step % STEPS_PER_HEAD) * HALF;
+#pragma unroll
+      for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int q = 0; q < HALF; ++q) {
+            if (rowok[m][h]) a[m][h][q] = ld_stream16(rowp[m][h] + int64_t(g) * p.kv_sh + 32 * (kk0 + q));
+            else a[m][h][q] = make_uint4(0u, 0u, 0u, 0u);
+          }
+    };
+    const int n_steps = g_count * STEPS_PER_HEAD;
+    uint4 cur[2][2][HALF], nxt[2][2][HALF];
+    load_step(0, cur);
+    for (int step = 0; step < n_steps; ++step) {
+      if (step + 1 < n_steps) load_step(step + 1, nxt);
+      const int g = g_first + step / STEPS_PER_HEAD;
+      const int kk0 = (step % STEPS_PER_HEAD) * HALF;
+      // The tensor core adds into its accumulator with truncation, which over the ~1500 chained
+      // products of a joint row would bias the sum by a visible fraction of an fp16 ulp.  So a
+      // chain inside the tensor core covers only one 32-channel block (6 products); the running
+      // sums are kept outside, in round-to-nearest fp32 adds.
+#pragma unroll
+      for (int q = 0; q < HALF; ++q) {
+        const uint2* bf = bfrag + (int64_t(g * KS + 2 * (kk0 + q)) * NT * 3) * 32 + lane;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float tmp[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+          for (int sub = 0; sub < 2; ++sub)
+#pragma unroll
+            for (int pc = 0; pc < 3; ++pc) {
+              const uint2 bb = bf[((sub * NT + nt) * 3 + pc) * 32];
+#pragma unroll
+              for (int m = 0; m < 2; ++m) {
+                const uint4 lo = cur[m][0][q], hi = cur[m][1][q];   // rows g8 and g8 + 8
+                mma_bf16_16816(tmp[m], sub ? lo.z : lo.x, sub ? hi.z : hi.x, sub ? lo.w : lo.y, sub ? hi.w : hi.y,
+                               bb.x, bb.y);
+              }
+            }
+#pragma unroll
+          for (int m = 0; m < 2; ++m)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[m][nt][e] += tmp[m][e];
+        }
+      }
+#pragma unroll
+      for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int q = 0; q < HALF; ++q) cur[m][h][q] = nxt[m][h][q];
+    }
+    // ---- one rounding into the metadata type -------------------------------------------------------
+    META_T* Mo = meta + int64_t(b) * p.meta_sb + int64_t(hm) * p.meta_sh;
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (!rowok[m][h]) continue;
+        const int n = n0 + 16 * m + 8 * h + g8;
+        META_T* row = Mo + int64_t(n) * p.meta_sn + 2 * t4;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const float x = acc[m][nt][2 * h], y = acc[m][nt][2 * h + 1];
+          if constexpr (sizeof(META_T) == 2) *reinterpret_cast<__half2*>(row + nt * 8) = __floats2half2_rn(x, y);
+          else *reinterpret_cast<float2*>(row + nt * 8) = make_float2(x, y);
+        }
+      }
+  }
+}
+
+template <typename META_T, int D, int NT>
+cudaError_t launch_mma_one(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
+                           cudaStream_t st) {
+  const size_t smem = size_t(p.Hkv) * (D / 16) * NT * 3 * 32 * sizeof(uint2);
+  auto kern = project_keys_mma_kernel<META_T, D, NT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+  if (e != cudaSuccess) return e;
+  const int tiles_per_row = (n_end - n_begin + 31) / 32;
+  const int64_t items = int64_t(p.B) * p.Hm * tiles_per_row;
+  const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(kNumSMs, (items + kMmaWarps - 1) / kMmaWarps)));
+  kern<<<ctas, kMmaWarps * 32, smem, st>>>(p, static_cast<const __nv_bfloat16*>(K), proj, static_cast<META_T*>(meta),
+                                           n_begin, n_end, tiles_per_row);
+  return cudaGetLastError();
+}
+
+// True (and launched) when the tensor-core path covers the problem.
+template <typename META_T>
+bool try_launch_mma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
+                    cudaStream_t st, cudaError_t* err) {
+  if (p.kv_dtype != KVSWAP_BF16 || (p.r != 16 && p.r != 32 && p.r != 64)) return false;
+  const size_t smem = size_t(p.Hkv) * (p.d / 16) * (p.r / 8) * 3 * 32 * sizeof(uint2);
+  if (smem > 200 * 1024) return false;
+  if (p.d == 128) {
+    if (p.r == 16) *err = launch_mma_one<META_T, 128, 2>(p, K, proj, meta, n_begin, n_end, st);
+    else if (p.r == 32) *err = launch_mma_one<META_T, 128, 4>(p, K, proj, meta, n_begin, n_end, st);
+    else *err = launch_mma_one<META_T, 128, 8>(p, K, proj, meta, n_begin, n_end, st);
+  } else {
+    if (p.r == 16) *err = launch_mma_one<META_T, 64, 2>(p, K, proj, meta, n_begin, n_end, st);
+    else if (p.r == 32) *err = launch_mma_one<META_T, 64, 4>(p, K, proj, meta, n_begin, n_end, st);
+    else *err = launch_mma_one<META_T, 64, 8>(p, K, proj, meta, n_begin, n_end, st);
+  }
+  return true;
+}
+
 template <typename KV_T, typename META_T>
 cudaError_t dispatch_rc(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
                         cudaStream_t st) {
@@ -108,7 +318,12 @@ cudaError_t dispatch_rc(const Problem& p, const void* K, const float* proj, void
 template <typename KV_T>
 cudaError_t dispatch_meta(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
                           cudaStream_t st) {
-  if (p.meta_dtype == KVSWAP_F16) return dispatch_rc<KV_T, __half>(p, K, proj, meta, n_begin, n_end, st);
+  cudaError_t e = cudaSuccess;
+  if (p.meta_dtype == KVSWAP_F16) {
+    if (try_launch_mma<__half>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
+    return dispatch_rc<KV_T, __half>(p, K, proj, meta, n_begin, n_end, st);
+  }
+  if (try_launch_mma<float>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
   return dispatch_rc<KV_T, float>(p, K, proj, meta, n_begin, n_end, st);
 }
 
