@@ -49,10 +49,14 @@ lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restri
   for (int g = g0; g < g1; ++g) {
     __syncthreads();
     for (int c = threadIdx.x; c < p.d; c += kThreads) {
+      // the rho loads are independent: issue them four at a time (one memory round trip for rho <= 4)
+      const Q_T* qc = q + (int64_t(b) * p.Hq + g * p.rho) * p.d + c;
       float s = 0.f;
-      for (int hh = 0; hh < p.rho; ++hh) {
-        const Q_T v = q[(int64_t(b) * p.Hq + g * p.rho + hh) * p.d + c];
-        if constexpr (sizeof(Q_T) == 4) s += v; else s += float(v);
+      for (int h0 = 0; h0 < p.rho; h0 += 4) {
+        float v[4];
+#pragma unroll
+        for (int hh = 0; hh < 4; ++hh) v[hh] = (h0 + hh < p.rho) ? float(qc[int64_t(h0 + hh) * p.d]) : 0.f;
+        s += (v[0] + v[1]) + (v[2] + v[3]);
       }
       qsum[c] = s;
     }
