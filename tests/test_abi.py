@@ -83,8 +83,8 @@ def test_entry_points_reject_null_and_small_workspace_without_touching_the_gpu(l
 
 
 def test_status_strings_and_version(lib):
-    seen = {kv.status_string(i) for i in range(9)}
-    assert len(seen) == 9 and "ok" in seen
+    seen = {kv.status_string(i) for i in range(11)}
+    assert len(seen) == 11 and "ok" in seen
     assert kv.status_string(123) == "unknown status"
     assert kv.kvswap_version() >= 100
 
@@ -93,3 +93,15 @@ def test_workspace_grows_with_the_problem(lib):
     small = kv.kvswap_workspace_bytes(good_shape())
     big = kv.kvswap_workspace_bytes(good_shape(batch=8, n_ctx=65536))
     assert big > small
+
+
+def test_device_status_entry_points_validate_their_arguments(lib):
+    assert lib.kvswap_workspace_init(None, 1024, None) == 1            # NULL workspace
+    assert lib.kvswap_workspace_init(ctypes.c_void_p(4096), 16, None) == 5   # shorter than the header
+    assert lib.kvswap_read_device_status(None, None) == 1
+
+
+def test_selected_token_count_is_bounded(lib):
+    """top_k * group_size beyond 2^30 is refused instead of overflowing the token arithmetic."""
+    assert kv.kvswap_validate_shape(good_shape(top_k=1 << 29, group_size=4)) == 6
+    assert kv.kvswap_validate_shape(good_shape(top_k=1 << 28, group_size=4)) == 0

@@ -303,3 +303,17 @@ def test_calls_run_on_a_side_stream():
     check_selection(R, dl.idx.cpu().numpy(), dl.nsel.cpu().numpy(), li.wl.top_k)
     out_o, _ = O.attend(li.q, li.K, li.V, dl.idx.cpu().numpy()[:, :, :li.wl.top_k], li.wl.group_size)
     assert np.abs(dl.out.cpu().numpy() - out_o).max() <= 1e-5
+
+
+def test_device_status_word_round_trip():
+    """The status word lives in the first bytes of the workspace: cleared by kvswap_workspace_init,
+    reported by kvswap_read_device_status (a non-zero word reads as KVSWAP_ERR_TIMEOUT).  No wait is
+    made to fail here: the word is poked from the host side."""
+    shape = rt.shape_for(W.CONFIGS[1], 1)
+    ws = rt.alloc_workspace(shape)
+    assert kv.kvswap_read_device_status(ws) == 0
+    ws[:4] = torch.tensor([1, 0, 0, 0], dtype=torch.uint8, device="cuda")
+    assert kv.kvswap_read_device_status(ws) == 10
+    assert "wait" in kv.status_string(10)
+    kv.kvswap_workspace_init(ws)
+    assert kv.kvswap_read_device_status(ws) == 0
