@@ -148,11 +148,11 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rq = lane >> 2, qt = lane & 3;          // row within a read, quarter of the row
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kWarps * kDepth; ++s) mbar_init(smem_addr(&ctl->full[s]), 1);
+  if (lane == 0) {                                  // every warp sets up its own stages: no CTA-wide wait
+    for (int s = 0; s < kDepth; ++s) mbar_init(smem_addr(&ctl->full[warp * kDepth + s]), 1);
     mbar_init_fence();
   }
-  __syncthreads();
+  __syncwarp();
 
   // Equal contiguous share of the work items for every warp of the grid (fewer than 2^31 items).
   const int rows_total = p.NG * p.G;                // scored rows per (sequence, metadata head)
@@ -342,28 +342,36 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rq = lane >> 2, qt = lane & 3;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kWarps * kDepth; ++s) mbar_init(smem_addr(&ctl->full[s]), 1);
+  if (lane == 0) {                                  // every warp sets up its own stages: no CTA-wide wait
+    for (int s = 0; s < kDepth; ++s) mbar_init(smem_addr(&ctl->full[warp * kDepth + s]), 1);
     mbar_init_fence();
   }
-  __syncthreads();
+  __syncwarp();
 
   const int rows_total = p.NG * p.G;
-  const int64_t items = int64_t(p.B) * n_sub * tiles_per_row;
+  const int hm_count = (p.Hm == 1) ? 1 : p.Hkv;   // per-head metadata: one scope (column 0) per head
+  const int64_t items = int64_t(p.B) * hm_count * n_sub * tiles_per_row;
   const int64_t gw = int64_t(blockIdx.x) * kWarps + warp, n_gw = int64_t(gridDim.x) * kWarps;
   const int first = int(items * gw / n_gw), last = int(items * (gw + 1) / n_gw);
   const int my_tiles = last - first;
-  int f_tile = first % tiles_per_row, f_rest = first / tiles_per_row;     // rest = b * n_sub + sub
+  int f_tile = first % tiles_per_row, f_rest = first / tiles_per_row;     // rest = (b * hm_count + hm) * n_sub + sub
   int c_tile = f_tile, c_rest = f_rest;
 
   const uint32_t ring = smem_addr(tiles) + uint32_t(warp) * kDepth * kTileBytes;
+  const __half* f_base = nullptr;                   // metadata of the fill cursor's (sequence, head)
+  int f_base_rest = -1;
   auto fill = [&](int stage) {
     if (lane == 0) {
+      if (f_rest != f_base_rest) {                  // divisions only when the cursor enters a new row set
+        f_base_rest = f_rest;
+        const int bh = f_rest / n_sub;
+        f_base = meta + int64_t(bh / hm_count) * p.meta_sb + int64_t(bh % hm_count) * p.meta_sh;
+      }
       const int rows = min(kTileRows, rows_total - f_tile * kTileRows);
-      const __half* src = meta + int64_t(f_rest / n_sub) * p.meta_sb + int64_t(f_tile) * kTileRows * p.meta_sn;
       const uint32_t bar = smem_addr(&ctl->full[warp * kDepth + stage]);
       mbar_arrive_expect_tx(bar, uint32_t(rows) * kRowBytes);
-      bulk_g2s(ring + uint32_t(stage) * kTileBytes, src, uint32_t(rows) * kRowBytes, bar);
+      bulk_g2s(ring + uint32_t(stage) * kTileBytes, f_base + int64_t(f_tile) * kTileRows * p.meta_sn,
+               uint32_t(rows) * kRowBytes, bar);
     }
     if (++f_tile == tiles_per_row) { f_tile = 0; ++f_rest; }
   };
@@ -374,7 +382,9 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
 
   uint32_t bhi[2][2], blo[2][2];                    // B fragments of k-steps 0 and 1
   float inv0 = 1.f, inv1 = 1.f;                     // undo the scaling of scopes 2t and 2t+1
-  int cur_rest = -1, b = 0, sub = 0;
+  int cur_rest = -1, b = 0, sub = 0, hm = 0;
+  float* out_row0 = scores;                         // scores row of the first scope of the current block
+  int ns_cur = 1;
   const int gb = (g_shift < 3) ? g_shift : 3;
   float run0 = -INFINITY, run1 = -INFINITY;         // running maxima of a 32-row group
   float* out = outbuf + warp * (NS * kOutStride);
@@ -385,11 +395,14 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
     const int tile = c_tile;
     if (c_rest != cur_rest) {                       // new (sequence, scope block): rebuild B
       cur_rest = c_rest;
-      sub = c_rest % n_sub; b = c_rest / n_sub;
-      const int sc = sub * NS + rq;                 // this lane supplies the query of scope sc
+      sub = c_rest % n_sub;
+      { const int bh = c_rest / n_sub; hm = bh % hm_count; b = bh / hm_count; }
+      // this lane supplies the query of column rq: scope sub * 8 + rq (joint) or head hm (column 0 only)
+      const int urow = (p.Hm == 1) ? sub * NS + rq : hm;
+      const bool have = (p.Hm == 1) ? (urow < p.S) : (rq == 0);
       float u[8];
-      if (sc < p.S) {
-        const float4* ur = reinterpret_cast<const float4*>(uq + (int64_t(b) * p.Su + sc) * p.r + qt * 8);
+      if (have) {
+        const float4* ur = reinterpret_cast<const float4*>(uq + (int64_t(b) * p.Su + urow) * p.r + qt * 8);
         const float4 x = ur[0], y = ur[1];
         u[0] = x.x; u[1] = x.y; u[2] = x.z; u[3] = x.w; u[4] = y.x; u[5] = y.y; u[6] = y.z; u[7] = y.w;
       } else {
@@ -420,6 +433,9 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
       }
       inv0 = __shfl_sync(kFull, inv, (2 * qt) * 4);
       inv1 = __shfl_sync(kFull, inv, (2 * qt + 1) * 4);
+      const int s0 = (p.Hm == 1) ? sub * NS : hm;
+      ns_cur = (p.Hm == 1) ? min(NS, p.S - s0) : 1;
+      out_row0 = scores + (int64_t(b) * p.S + s0) * p.NG;
     }
     if (++c_tile == tiles_per_row) { c_tile = 0; ++c_rest; }
     if (!__all_sync(kFull, mbar_wait(smem_addr(&ctl->full[warp * kDepth + stage]), phase))) { timed_out = true; break; }
@@ -473,12 +489,18 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
     }
     __syncwarp();
     {
-      const int g0 = (tile * kTileRows) >> g_shift;
-      const int s0 = sub * NS;
-      const int ns = min(NS, p.S - s0);
-      for (int i = lane; i < ns * ngt; i += 32) {
-        const int s = i / ngt, gi = i - s * ngt;
-        scores[(int64_t(b) * p.S + s0 + s) * p.NG + g0 + gi] = out[s * kOutStride + gi];
+      float* dst = out_row0 + ((tile * kTileRows) >> g_shift);
+      if (rows == kTileRows) {                      // full tile: 32 >> g_shift groups, a power of two
+        const int sh = 5 - g_shift;
+        for (int i = lane; i < (ns_cur << sh); i += 32) {
+          const int s = i >> sh, gi = i & ((1 << sh) - 1);
+          dst[int64_t(s) * p.NG + gi] = out[s * kOutStride + gi];
+        }
+      } else {
+        for (int i = lane; i < ns_cur * ngt; i += 32) {
+          const int s = i / ngt, gi = i - s * ngt;
+          dst[int64_t(s) * p.NG + gi] = out[s * kOutStride + gi];
+        }
       }
     }
     __syncwarp();
@@ -613,8 +635,8 @@ cudaError_t launch_mma(const Problem& p, const float* uq, const void* meta, floa
   constexpr int NS = 8;
   const int rows_total = p.NG * p.G;
   const int tiles_per_row = (rows_total + kTileRows - 1) / kTileRows;
-  const int n_sub = (p.S + NS - 1) / NS;
-  const int64_t items = int64_t(p.B) * n_sub * tiles_per_row;
+  const int n_sub = (p.Hm == 1) ? (p.S + NS - 1) / NS : 1;
+  const int64_t items = int64_t(p.B) * ((p.Hm == 1) ? 1 : p.Hkv) * n_sub * tiles_per_row;
   const int64_t want = (items + kWarps - 1) / kWarps;
   const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(2 * kNumSMs, want)));
   const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kOutStride;
@@ -635,9 +657,10 @@ cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, flo
                          tile_items < (int64_t(1) << 30);
   if (streaming) {
     const int ns = (p.Hm == 1) ? p.S : 1;
-    if constexpr (std::is_same<META_T, __half>::value) {
-      if (ns >= 3) return launch_mma(p, uq, meta, scores, g_shift, err, st);
-    }
+    // fp16 metadata: the tensor-core scorer serves every streaming case (with one score per
+    // row it uses one of its eight columns; it is still far cheaper in instructions per row
+    // than the fp32 pipes, which at one dot product per 64-byte row are issue-bound, not HBM-bound).
+    if constexpr (std::is_same<META_T, __half>::value) return launch_mma(p, uq, meta, scores, g_shift, err, st);
     if (ns == 1) return launch_tiles<META_T, 1>(p, uq, meta, scores, g_shift, err, st);
     if (ns == 2) return launch_tiles<META_T, 2>(p, uq, meta, scores, g_shift, err, st);
     if (ns <= 4) return launch_tiles<META_T, 4>(p, uq, meta, scores, g_shift, err, st);

@@ -23,6 +23,7 @@
 // What a warp does with a chunk is the business of its compute engine (below): fp32 pipes for
 // fp32 K/V, tensor cores for 16-bit K/V.
 #include <algorithm>
+#include <cstdint>
 
 #include "async_copy.cuh"
 #include "common.cuh"
@@ -669,19 +670,17 @@ void plan_sparse_decode(const Problem& p, Workspace* w) {
   const int64_t problems = int64_t(p.B) * p.Hkv * (p.rho / rh);
   const int64_t tokens = int64_t(p.M) * p.G + (p.N - int64_t(p.NG) * p.G);
   const int64_t n_chunks = std::max<int64_t>(1, (tokens + kTok - 1) / kTok);
-  // One wave of 2 CTAs per SM when the problems are few; otherwise the split that fills whole
-  // waves best, keeping at least two chunks per compute warp and split.
+  // Cost of a split factor s, in chunk times of the slowest CTA: waves * (chunks per CTA + the
+  // fixed part of a CTA -- first index fetch, first rows, merge -- worth about 14 chunks), with
+  // 2 CTAs per SM resident; at least two chunks per warp and split.
   const int64_t slots = int64_t(kNumSMs) * 2;
   const int64_t max_splits = std::min<int64_t>(256, std::max<int64_t>(1, n_chunks / (2 * kWarps)));
-  int64_t best = 1;
-  double best_eff = 0.0;
+  int64_t best = 1, best_cost = INT64_MAX;
   for (int64_t s = 1; s <= max_splits; ++s) {
-    const int64_t ctas = problems * s;
-    const int64_t waves = (ctas + slots - 1) / slots;
+    const int64_t waves = (problems * s + slots - 1) / slots;
     if (waves > 2 && s > 1) break;
-    const int64_t per = (n_chunks + s - 1) / s;               // chunks of the largest split
-    const double eff = double(n_chunks) * problems / (double(waves) * slots * per);
-    if (eff > best_eff * 1.02) { best_eff = eff; best = s; }
+    const int64_t cost = waves * ((n_chunks + s - 1) / s + 14);
+    if (cost < best_cost) { best_cost = cost; best = s; }
   }
   w->splits = int(best);
   const size_t row = size_t(p.d) * (p.kv_dtype == KVSWAP_F32 ? 4 : 2);
