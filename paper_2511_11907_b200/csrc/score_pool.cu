@@ -313,10 +313,11 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
 // products per k-step), so the only rounding is the accumulator's.
 //
 // Operand layout.  A 16-byte shared-memory read gives lane (g = lane / 4, t = lane % 4) the rank
-// entries 8t..8t+7 of row g.  The contraction index may be permuted freely as long as both
-// operands agree, so k-step j takes entries 8t+4j..8t+4j+3 as the four A values the lane owes for
-// its row, and the lane's B values are the same entries of the query of scope g.  The
-// accumulator then holds rows g and g+8 for scopes 2t and 2t+1.
+// entries 8t..8t+7 of row g of an 8-row block.  The contraction index may be permuted freely as
+// long as both operands agree, so k-step j takes entries 8t+4j..8t+4j+3 as the four values the
+// lane owes for token g (the column operand, 8 tokens wide), and the row operand holds the same
+// entries of the query of scope g (rows 8..15 are zero).  The accumulator then holds, in lane
+// (g, t), the scores of scope g for tokens 2t and 2t+1.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -330,10 +331,12 @@ __device__ __forceinline__ uint32_t pack_half2(__half lo, __half hi) {
   return uint32_t(__half_as_ushort(lo)) | (uint32_t(__half_as_ushort(hi)) << 16);
 }
 
+template <int GS>                                    // GS = log2(G), 0..5
 __global__ void __launch_bounds__(kWarps * 32, 2)
 score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __restrict__ meta,
-                      float* __restrict__ scores, int tiles_per_row, int n_sub, int g_shift,
+                      float* __restrict__ scores, int tiles_per_row, int n_sub,
                       uint32_t* __restrict__ err) {
+  constexpr int g_shift = GS;
   constexpr int NS = 8;
   extern __shared__ __align__(128) unsigned char dyn[];
   unsigned char* tiles = dyn;
@@ -380,13 +383,13 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
   pdl_wait();
   pdl_trigger();
 
-  uint32_t bhi[2][2], blo[2][2];                    // B fragments of k-steps 0 and 1
-  float inv0 = 1.f, inv1 = 1.f;                     // undo the scaling of scopes 2t and 2t+1
+  uint32_t bhi[2][2], blo[2][2];                    // query fragments (head, remainder) of k-steps 0 and 1
+  float inv = 1.f;                                  // undoes the scaling of this lane's scope
   int cur_rest = -1, b = 0, sub = 0, hm = 0;
   float* out_row0 = scores;                         // scores row of the first scope of the current block
   int ns_cur = 1;
-  const int gb = (g_shift < 3) ? g_shift : 3;
-  float run0 = -INFINITY, run1 = -INFINITY;         // running maxima of a 32-row group
+  constexpr int gb = (GS < 3) ? GS : 3;             // butterfly levels over the row bits
+  float run = -INFINITY;                            // running maximum of a 16- or 32-row group
   float* out = outbuf + warp * (NS * kOutStride);
   int stage = 0;
   uint32_t phase = 0;
@@ -418,7 +421,7 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
       int sh = 0;
       if (mx > 0.f && mx < INFINITY) sh = min(120, max(-113, 14 - (int((__float_as_uint(mx) >> 23) & 0xffu) - 127)));
       const float scale = __uint_as_float(uint32_t(sh + 127) << 23);
-      const float inv = __uint_as_float(uint32_t(127 - sh) << 23);
+      inv = __uint_as_float(uint32_t(127 - sh) << 23);
       __half hi[8], lo[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -431,8 +434,6 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
         bhi[j][0] = pack_half2(hi[4 * j], hi[4 * j + 1]); bhi[j][1] = pack_half2(hi[4 * j + 2], hi[4 * j + 3]);
         blo[j][0] = pack_half2(lo[4 * j], lo[4 * j + 1]); blo[j][1] = pack_half2(lo[4 * j + 2], lo[4 * j + 3]);
       }
-      inv0 = __shfl_sync(kFull, inv, (2 * qt) * 4);
-      inv1 = __shfl_sync(kFull, inv, (2 * qt + 1) * 4);
       const int s0 = (p.Hm == 1) ? sub * NS : hm;
       ns_cur = (p.Hm == 1) ? min(NS, p.S - s0) : 1;
       out_row0 = scores + (int64_t(b) * p.S + s0) * p.NG;
@@ -442,47 +443,39 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
     const int rows = min(kTileRows, rows_total - tile * kTileRows);
     const int ngt = rows >> g_shift;                // groups in this tile
     const uint32_t base = ring + uint32_t(stage) * kTileBytes + uint32_t(lane) * 16u;
+    // Scopes are the row operand (rows 8..15 unused), 8 tokens the column operand: lane (g, t)
+    // receives the scores of scope g for tokens 2t and 2t+1 of each 8-row read, so a group's
+    // maximum is a max over two registers and at most two shuffles.
+    const bool scope_ok = rq < ns_cur;
+    float* orow = out + rq * kOutStride;
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      if (mt * 16 < rows) {
-        uint32_t wa[4], wb[4];                      // rows g and g + 8 of this 16-row block
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(wa[0]), "=r"(wa[1]), "=r"(wa[2]), "=r"(wa[3])
-                     : "r"(base + uint32_t(mt) * 16u * kRowBytes));
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(wb[0]), "=r"(wb[1]), "=r"(wb[2]), "=r"(wb[3])
-                     : "r"(base + uint32_t(mt) * 16u * kRowBytes + 8u * kRowBytes));
+    for (int it = 0; it < kTileRows / 8; ++it) {
+      if (it * 8 < rows) {
+        uint32_t w[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
+                     : "r"(base + uint32_t(it) * 8u * kRowBytes));
         float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-          mma16816(d, wa[2 * j], wb[2 * j], wa[2 * j + 1], wb[2 * j + 1], bhi[j][0], bhi[j][1]);
-          mma16816(d, wa[2 * j], wb[2 * j], wa[2 * j + 1], wb[2 * j + 1], blo[j][0], blo[j][1]);
+          mma16816(d, bhi[j][0], 0u, bhi[j][1], 0u, w[2 * j], w[2 * j + 1]);
+          mma16816(d, blo[j][0], 0u, blo[j][1], 0u, w[2 * j], w[2 * j + 1]);
         }
-        float x0 = d[0] * inv0, x1 = d[1] * inv1;   // row g,     scopes 2t, 2t+1
-        float y0 = d[2] * inv0, y1 = d[3] * inv1;   // row g + 8, scopes 2t, 2t+1
-        if (g_shift >= 4) { x0 = fmaxf(x0, y0); x1 = fmaxf(x1, y1); }
-        if (gb >= 1) {
-          x0 = fmaxf(x0, __shfl_xor_sync(kFull, x0, 4)); x1 = fmaxf(x1, __shfl_xor_sync(kFull, x1, 4));
-          y0 = fmaxf(y0, __shfl_xor_sync(kFull, y0, 4)); y1 = fmaxf(y1, __shfl_xor_sync(kFull, y1, 4));
-        }
-        if (gb >= 2) {
-          x0 = fmaxf(x0, __shfl_xor_sync(kFull, x0, 8)); x1 = fmaxf(x1, __shfl_xor_sync(kFull, x1, 8));
-          y0 = fmaxf(y0, __shfl_xor_sync(kFull, y0, 8)); y1 = fmaxf(y1, __shfl_xor_sync(kFull, y1, 8));
-        }
-        if (gb >= 3) {
-          x0 = fmaxf(x0, __shfl_xor_sync(kFull, x0, 16)); x1 = fmaxf(x1, __shfl_xor_sync(kFull, x1, 16));
-          y0 = fmaxf(y0, __shfl_xor_sync(kFull, y0, 16)); y1 = fmaxf(y1, __shfl_xor_sync(kFull, y1, 16));
-        }
-        if ((rq & ((1 << gb) - 1)) == 0) {          // lanes of a group's first row publish it
-          float* o0 = out + (2 * qt) * kOutStride;
-          float* o1 = o0 + kOutStride;
-          if (g_shift <= 3) {
-            const int gx = (mt * 16 + rq) >> g_shift, gy = (mt * 16 + 8 + rq) >> g_shift;
-            if (gx < ngt) { o0[gx] = x0; o1[gx] = x1; }
-            if (gy < ngt) { o0[gy] = y0; o1[gy] = y1; }
-          } else if (g_shift == 4) {
-            o0[mt] = x0; o1[mt] = x1;
-          } else {                                  // G = 32: the tile is one group
-            run0 = fmaxf(run0, x0); run1 = fmaxf(run1, x1);
-            if (mt == 1) { o0[0] = run0; o1[0] = run1; run0 = -INFINITY; run1 = -INFINITY; }
+        const float x0 = d[0] * inv, x1 = d[1] * inv;            // tokens 2t and 2t+1 of this read
+        if constexpr (GS == 0) {
+          if (scope_ok) { orow[it * 8 + 2 * qt] = x0; orow[it * 8 + 2 * qt + 1] = x1; }
+        } else {
+          float m = fmaxf(x0, x1);
+          if constexpr (GS >= 2) m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
+          if constexpr (GS >= 3) m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
+          if constexpr (GS == 1) { if (scope_ok) orow[it * 4 + qt] = m; }
+          else if constexpr (GS == 2) { if (scope_ok && (qt & 1) == 0) orow[it * 2 + (qt >> 1)] = m; }
+          else if constexpr (GS == 3) { if (scope_ok && qt == 0) orow[it] = m; }
+          else {                                                 // G = 16 or 32: 2 or 4 reads per group
+            run = fmaxf(run, m);
+            if (((it + 1) & ((1 << (GS - 3)) - 1)) == 0) {
+              if (scope_ok && qt == 0) orow[it >> (GS - 3)] = run;
+              run = -INFINITY;
+            }
           }
         }
       }
@@ -640,10 +633,20 @@ cudaError_t launch_mma(const Problem& p, const float* uq, const void* meta, floa
   const int64_t want = (items + kWarps - 1) / kWarps;
   const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(2 * kNumSMs, want)));
   const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kOutStride;
-  cudaError_t e = cudaFuncSetAttribute(score_pool_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-  if (e != cudaSuccess) return e;
-  return launch_pdl(score_pool_mma_kernel, dim3(ctas), dim3(kWarps * 32), smem, st, p, uq,
-                    static_cast<const __half*>(meta), scores, tiles_per_row, n_sub, g_shift, err);
+  auto go = [&](auto kern) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (e != cudaSuccess) return e;
+    return launch_pdl(kern, dim3(ctas), dim3(kWarps * 32), smem, st, p, uq, static_cast<const __half*>(meta), scores,
+                      tiles_per_row, n_sub, err);
+  };
+  switch (g_shift) {
+    case 0: return go(score_pool_mma_kernel<0>);
+    case 1: return go(score_pool_mma_kernel<1>);
+    case 2: return go(score_pool_mma_kernel<2>);
+    case 3: return go(score_pool_mma_kernel<3>);
+    case 4: return go(score_pool_mma_kernel<4>);
+    default: return go(score_pool_mma_kernel<5>);
+  }
 }
 
 template <typename META_T>
