@@ -332,7 +332,7 @@ __device__ __forceinline__ uint32_t pack_half2(__half lo, __half hi) {
 }
 
 template <int GS>                                    // GS = log2(G), 0..5
-__global__ void __launch_bounds__(kWarps * 32, 2)
+__global__ void __launch_bounds__(kWarps * 32, 3)
 score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __restrict__ meta,
                       float* __restrict__ scores, int tiles_per_row, int n_sub,
                       uint32_t* __restrict__ err) {
@@ -631,7 +631,10 @@ cudaError_t launch_mma(const Problem& p, const float* uq, const void* meta, floa
   const int n_sub = (p.Hm == 1) ? (p.S + NS - 1) / NS : 1;
   const int64_t items = int64_t(p.B) * ((p.Hm == 1) ? 1 : p.Hkv) * n_sub * tiles_per_row;
   const int64_t want = (items + kWarps - 1) / kWarps;
-  const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(2 * kNumSMs, want)));
+  // Three CTAs per SM hide the per-tile bookkeeping better, but only pay when every warp still has
+  // a fair number of tiles; short streams run as one wave of two per SM.
+  const int per_sm = (items >= int64_t(10) * 2 * kNumSMs * kWarps) ? 3 : 2;
+  const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(per_sm * kNumSMs, want)));
   const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kOutStride;
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
