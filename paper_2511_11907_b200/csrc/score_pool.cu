@@ -31,40 +31,47 @@ constexpr uint32_t kFull = 0xffffffffu;
 // contraction index x 32 output columns (r <= 32), or the generic loop for larger r.
 // ------------------------------------------------------------------------------------------
 template <typename Q_T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(4 * kThreads)
 lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restrict__ proj,
                      float* __restrict__ uq) {
-  __shared__ float qsum[128];
-  __shared__ float red[kThreads];
+  // blockDim.x = kThreads * n_grp: thread group `grp` (256 threads) takes the KV heads
+  // g0 + grp, g0 + grp + n_grp, ... of the row, so that up to four heads are in flight at once.
+  __shared__ float qsum[4][128];
+  __shared__ float red[4 * kThreads];
   pdl_wait();
   pdl_trigger();
   const int b = blockIdx.x, row = blockIdx.y;
+  const int tid = threadIdx.x % kThreads, grp = threadIdx.x / kThreads, n_grp = blockDim.x / kThreads;
   // KV heads summed into this row
   const bool joint_all = (p.Hm == 1 && p.scope == KVSWAP_SCOPE_ALL_HEADS);
   const int g0 = joint_all ? 0 : row;
   const int g1 = joint_all ? p.Hkv : row + 1;
   const int parts = kThreads / p.r;               // r <= 256
-  const int j = threadIdx.x % p.r, part = threadIdx.x / p.r;
+  const int j = tid % p.r, part = tid / p.r;
   float acc = 0.f;
-  for (int g = g0; g < g1; ++g) {
+  for (int gb = g0; gb < g1; gb += n_grp) {       // every group runs every iteration (barriers inside)
+    const int g = gb + grp;
+    const bool on = g < g1;
     __syncthreads();
-    for (int c = threadIdx.x; c < p.d; c += kThreads) {
-      // the rho loads are independent: issue them four at a time (one memory round trip for rho <= 4)
-      const Q_T* qc = q + (int64_t(b) * p.Hq + g * p.rho) * p.d + c;
-      float s = 0.f;
-      for (int h0 = 0; h0 < p.rho; h0 += 4) {
-        float v[4];
+    if (on) {
+      for (int c = tid; c < p.d; c += kThreads) {
+        // the rho loads are independent: issue them four at a time (one memory round trip for rho <= 4)
+        const Q_T* qc = q + (int64_t(b) * p.Hq + g * p.rho) * p.d + c;
+        float s = 0.f;
+        for (int h0 = 0; h0 < p.rho; h0 += 4) {
+          float v[4];
 #pragma unroll
-        for (int hh = 0; hh < 4; ++hh) v[hh] = (h0 + hh < p.rho) ? float(qc[int64_t(h0 + hh) * p.d]) : 0.f;
-        s += (v[0] + v[1]) + (v[2] + v[3]);
+          for (int hh = 0; hh < 4; ++hh) v[hh] = (h0 + hh < p.rho) ? float(qc[int64_t(h0 + hh) * p.d]) : 0.f;
+          s += (v[0] + v[1]) + (v[2] + v[3]);
+        }
+        qsum[grp][c] = s;
       }
-      qsum[c] = s;
     }
     // The adapter rows do not depend on q: fetch this thread's share before the barrier.
-    const float* Pg = proj + int64_t(g) * p.d * p.r;
+    const float* Pg = proj + int64_t(on ? g : g0) * p.d * p.r;
     float pj[16];
     int n_c = 0;
-    if (part < parts) {
+    if (on && part < parts) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const int c = part + i * parts;
@@ -73,15 +80,15 @@ lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restri
       n_c = (p.d - part + parts - 1) / parts;
     }
     __syncthreads();
-    if (part < parts) {
+    if (on && part < parts) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const int c = part + i * parts;
-        if (c < p.d) acc = fmaf(qsum[c], pj[i], acc);
+        if (c < p.d) acc = fmaf(qsum[grp][c], pj[i], acc);
       }
       for (int i = 16; i < n_c; ++i) {              // only when d / parts > 16 (large r)
         const int c = part + i * parts;
-        acc = fmaf(qsum[c], Pg[int64_t(c) * p.r + j], acc);
+        acc = fmaf(qsum[grp][c], Pg[int64_t(c) * p.r + j], acc);
       }
     }
   }
@@ -89,7 +96,8 @@ lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restri
   __syncthreads();
   if (threadIdx.x < p.r) {
     float s = 0.f;
-    for (int k = 0; k < parts; ++k) s += red[k * p.r + threadIdx.x];
+    for (int gq = 0; gq < n_grp; ++gq)
+      for (int k = 0; k < parts; ++k) s += red[gq * kThreads + k * p.r + threadIdx.x];
     uq[(int64_t(b) * p.Su + row) * p.r + threadIdx.x] = s;
   }
 }
@@ -686,14 +694,18 @@ cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, flo
 
 cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* proj, float* uq, cudaStream_t st) {
   dim3 grid(p.B, p.Su);
+  // One 256-thread group per KV head in flight: one group per row, up to four when a row sums
+  // all KV heads (joint metadata under the all-heads scope).
+  const bool joint_all = (p.Hm == 1 && p.scope == KVSWAP_SCOPE_ALL_HEADS);
+  const dim3 block(kThreads * (joint_all ? std::min(4, p.Hkv) : 1));
   switch (p.q_dtype) {
     case KVSWAP_F32:
-      return launch_pdl(lowrank_query_kernel<float>, grid, dim3(kThreads), 0, st, p, static_cast<const float*>(q), proj, uq);
+      return launch_pdl(lowrank_query_kernel<float>, grid, block, 0, st, p, static_cast<const float*>(q), proj, uq);
     case KVSWAP_BF16:
-      return launch_pdl(lowrank_query_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, st, p,
+      return launch_pdl(lowrank_query_kernel<__nv_bfloat16>, grid, block, 0, st, p,
                         static_cast<const __nv_bfloat16*>(q), proj, uq);
     default:
-      return launch_pdl(lowrank_query_kernel<__half>, grid, dim3(kThreads), 0, st, p, static_cast<const __half*>(q), proj, uq);
+      return launch_pdl(lowrank_query_kernel<__half>, grid, block, 0, st, p, static_cast<const __half*>(q), proj, uq);
   }
 }
 
