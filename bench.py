@@ -33,10 +33,11 @@ from paper_2511_11907_b200 import workloads as W  # noqa: E402
 METRIC = "decode_steps_per_sec"
 UNIT = "steps/s"
 
-# DRAM bytes (read + write) per launch of the split-K sparse-decode kernel, from the ncu capture
-# summarised in profiles/sparse_decode_config5_one_layer.md; None for workloads not captured.
-# Key: (config, metadata layout, scope).
-NCU_TRAFFIC = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the split-K sparse-decode
+# kernel, from the ncu capture summarised in profiles/decode_kernels_config5_one_layer.md (taken at
+# full config-5 shapes on one layer; the traffic of a launch does not depend on the layer count).
+# None for workloads that were not captured.  Key: (config, metadata layout, scope).
+NCU_TRAFFIC = {(5, "joint", "kv_head"): 134444800 + 4012032}
 
 
 def parse_args():

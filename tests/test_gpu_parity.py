@@ -166,6 +166,28 @@ EDGE = {
     "rank_24_fp32": small(rank=24),
     "rank_64": small(rank=64, head_dim=128),
     "several_tiles": small(n_ctx=5000 + 2, group_size=8, top_k=100, batch=1),
+    # 16-bit K/V and fp16 metadata of 64-byte rows: the tensor-core scorer for every group size, more
+    # than 8 scopes, and the tensor-core attention engine for 2..4 heads per K/V row, both 16-bit types
+    "f16meta_group_1": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=1,
+                             n_ctx=700, top_k=40),
+    "f16meta_group_2": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=2,
+                             n_ctx=2 * 333 + 1, top_k=25),
+    "f16meta_group_4_rho_2": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32,
+                                   group_size=4, n_q_heads=4, n_kv_heads=2, n_ctx=4 * 257 + 2, top_k=30),
+    "f16meta_group_32": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32,
+                              group_size=32, n_ctx=32 * 41 + 9, top_k=7),
+    "f16meta_group_3_bf16": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32,
+                                  group_size=3, n_ctx=3 * 211 + 2, top_k=33),
+    "f16meta_twelve_scopes": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=64, rank=32,
+                                   group_size=8, n_q_heads=24, n_kv_heads=12, batch=1, n_ctx=8 * 150 + 5, top_k=20),
+    "fp16_kv_fp16_q": small(kv_dtype=W.F16, q_dtype=W.F16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=8,
+                            n_q_heads=6, n_kv_heads=2, n_ctx=8 * 90 + 3, top_k=12),
+    "bf16_rank_64": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=64, group_size=8,
+                          n_ctx=8 * 64 + 1, top_k=10),
+    # long score rows: 16 keys per thread in the register top-k, and the shared-memory top-k beyond it
+    "ten_thousand_groups": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=64, rank=32,
+                                 group_size=4, batch=1, n_ctx=4 * 10000 + 3, top_k=700),
+    "twenty_thousand_groups": small(group_size=1, batch=1, n_ctx=20000, top_k=1500),
 }
 
 
