@@ -66,6 +66,7 @@ void plan_workspace(const Problem& p, Workspace* w) {
   w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
   w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * std::max(p.NG, 1));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
+  w->off_adapter = off;  off += align256(project_keys_umma_scratch_bytes(p) + 1024);   // 1 KiB: tensor-map base alignment
   w->total = off;
 }
 
@@ -92,7 +93,6 @@ int kvswap_validate_shape(const kvswap_shape* shape) {
 
 int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* proj, void* meta_out,
                         int32_t n_begin, int32_t n_end, void* ws, size_t ws_bytes, void* cuda_stream) {
-  (void)ws; (void)ws_bytes;
   Problem p;
   int st = resolve(shape, &p);
   if (st != KVSWAP_OK) return st;
@@ -100,7 +100,21 @@ int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* p
   if (misaligned(K) || misaligned(proj) || misaligned(meta_out)) return KVSWAP_ERR_ALIGN;
   if (n_begin < 0 || n_end < n_begin || n_end > p.N) return KVSWAP_ERR_SHAPE;
   if (n_begin == n_end) return KVSWAP_OK;
-  cudaError_t e = launch_project_keys(p, K, proj, meta_out, n_begin, n_end, static_cast<cudaStream_t>(cuda_stream));
+  // The workspace is optional here: with one of at least kvswap_workspace_bytes() the bf16 / r = 32 /
+  // d = 128 case runs on tcgen05 (it needs room for the split adapter), otherwise on the warp-level path.
+  void* scratch = nullptr;
+  uint32_t* err = nullptr;
+  if (ws != nullptr && !misaligned(ws)) {
+    Workspace w;
+    plan_workspace(p, &w);
+    if (ws_bytes >= w.total) {
+      char* a = static_cast<char*>(ws) + w.off_adapter;
+      scratch = reinterpret_cast<void*>((reinterpret_cast<uintptr_t>(a) + 1023) & ~uintptr_t(1023));
+      err = static_cast<uint32_t*>(ws);
+    }
+  }
+  cudaError_t e = launch_project_keys(p, K, proj, meta_out, n_begin, n_end, scratch, err,
+                                      static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 

@@ -32,6 +32,7 @@ struct Workspace {
   size_t off_uq;       // float [B, Su, r]       summed low-rank queries
   size_t off_scores;   // float [B, S, NG]       group scores R (when the caller passes no buffer)
   size_t off_partial;  // float [B, Hq, splits, d + 2]  split-K partials (m, l, acc[d])
+  size_t off_adapter;  // bf16 [H_kv, 3 r, d]       adapter split into three bf16 pieces (project_keys on tcgen05)
   size_t total;
   int splits;          // split-K factor of sparse_decode for this shape
   int heads_per_cta;   // query heads sharing one K/V pass in sparse_decode
@@ -43,8 +44,12 @@ void plan_workspace(const Problem& p, Workspace* w);
 void plan_sparse_decode(const Problem& p, Workspace* w);   // fills splits, heads_per_cta, depth
 
 // Kernel launchers (each returns a cudaError_t from the launch).
+// `scratch` is the workspace region at off_adapter (project_keys_umma_scratch_bytes, may be NULL).
 cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta,
-                                int n_begin, int n_end, cudaStream_t st);
+                                int n_begin, int n_end, void* scratch, uint32_t* err, cudaStream_t st);
+size_t project_keys_umma_scratch_bytes(const Problem& p);
+bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
+                                  int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result);
 cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* proj, float* uq,
                                  cudaStream_t st);
 cudaError_t launch_score_pool(const Problem& p, const float* uq, const void* meta, float* scores,

@@ -330,7 +330,9 @@ cudaError_t dispatch_meta(const Problem& p, const void* K, const float* proj, vo
 }  // namespace
 
 cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
-                                int n_end, cudaStream_t st) {
+                                int n_end, void* scratch, uint32_t* err, cudaStream_t st) {
+  cudaError_t e = cudaSuccess;
+  if (try_launch_project_keys_umma(p, K, proj, meta, n_begin, n_end, scratch, err, st, &e)) return e;
   switch (p.kv_dtype) {
     case KVSWAP_F32: return dispatch_meta<float>(p, K, proj, meta, n_begin, n_end, st);
     case KVSWAP_BF16: return dispatch_meta<__nv_bfloat16>(p, K, proj, meta, n_begin, n_end, st);

@@ -1,0 +1,316 @@
+// K1 on the 5th-generation tensor cores: metadata build K_lr = Flatten(K) A (Sec. 4.2) with
+// tcgen05.mma, accumulators in tensor memory and operands staged by TMA.
+//
+// Covers bf16 K with d = 128 and r = 32 (the benchmark shapes); project_keys.cu keeps the
+// warp-level path for everything else.
+//
+// The adapter stays fp32-exact: every entry is split into three bf16 pieces, laid out by a small
+// preparation kernel as a K-major [3r x d] operand per KV head, so one instruction shape
+// M = 128 tokens, N = 96 = 3 x 32 columns, K = 16 channels yields the three partial products side
+// by side; the epilogue adds them in fp32.  The tensor core adds into its accumulator with
+// truncation, so a chain inside tensor memory covers one KV head (8 instructions); the sum over
+// the heads of a joint row is kept in registers with round-to-nearest adds.
+//
+// CTA = 6 warps, persistent (one per SM):
+//   warp 0   producer: per (token tile, KV head) two TMA boxes of K (128 rows x 64 channels,
+//            128-byte swizzle) and two of the split adapter into a ring of stages;
+//   warp 1   issues the MMAs (one thread), owns the tensor-memory allocation (two accumulators);
+//   warps 2-5 epilogue: tcgen05.ld of the finished accumulator (one token row per thread), sum of
+//            the three pieces, running sum over heads, one rounding into the metadata type.
+// Stages and accumulators are handed over through mbarriers; every wait is bounded.
+#include <cuda.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "async_copy.cuh"
+#include "common.cuh"
+
+namespace kvswap {
+namespace {
+
+constexpr int kD = 128, kR = 32, kNcols = 3 * kR;          // channels, rank, accumulator columns
+constexpr int kTileM = 128;                                // tokens per tile
+constexpr int kStages = 3;
+constexpr uint32_t kAHalf = kTileM * 128;                  // 128 rows x 128 bytes (64 bf16 channels)
+constexpr uint32_t kBHalf = kNcols * 128;
+constexpr uint32_t kStageBytes = 2 * kAHalf + 2 * kBHalf;  // 57344
+constexpr int kThreadsUmma = 6 * 32;
+constexpr uint32_t kTmemCols = 256;                        // two accumulators of 96 columns, at 0 and 128
+
+// ---- the adapter as three bf16 pieces, [g][piece * r + j][c] (K-major rows of d channels) ----------
+__global__ void split_adapter_kernel(const float* __restrict__ proj, __nv_bfloat16* __restrict__ bsplit, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;     // over [g][c][j]
+  if (i >= n) return;
+  const int j = i % kR, c = (i / kR) % kD, g = i / (kR * kD);
+  const float v = proj[i];
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+  __nv_bfloat16* dst = bsplit + (int64_t(g) * kNcols + j) * kD + c;
+  dst[0] = hi; dst[int64_t(kR) * kD] = mid; dst[int64_t(2 * kR) * kD] = lo;
+}
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_byte_addr) {
+  return uint64_t((smem_byte_addr >> 4) & 0x3fffu) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) |
+         (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+struct UmmaShared {
+  unsigned long long full[kStages];        // stage loaded (TMA bytes)
+  unsigned long long empty[kStages];       // stage consumed (MMA commit)
+  unsigned long long acc_full[2];          // accumulator finished (MMA commit)
+  unsigned long long acc_empty[2];         // accumulator read out (4 epilogue warps)
+  uint32_t tmem_base;
+  uint32_t abort;
+};
+
+template <typename META_T>
+__global__ void __launch_bounds__(kThreadsUmma, 1)
+project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_b,
+                         META_T* __restrict__ meta, int n_begin, int n_end, int tiles_per_row,
+                         uint32_t* __restrict__ err) {
+  extern __shared__ unsigned char dyn_raw[];
+  const uint32_t stage0 = (smem_addr(dyn_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
+  __shared__ UmmaShared sh;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_addr(&sh.full[s]), 1); mbar_init(smem_addr(&sh.empty[s]), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(smem_addr(&sh.acc_full[a]), 1); mbar_init(smem_addr(&sh.acc_empty[a]), 4); }
+    sh.abort = 0;
+    mbar_init_fence();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&sh.tmem_base)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  // Work: contiguous range of (sequence, metadata head, token tile) items; a step = (item, KV head).
+  const int g_count = (p.Hm == 1) ? p.Hkv : 1;
+  const int64_t items = int64_t(p.B) * p.Hm * tiles_per_row;
+  const int64_t first = items * blockIdx.x / gridDim.x, last = items * (blockIdx.x + 1) / gridDim.x;
+  const int n_steps = int(last - first) * g_count;
+
+  if (warp == 0) {
+    // ================================ producer ==============================================
+    if (lane == 0) {
+      for (int s = 0; s < n_steps; ++s) {
+        const int stage = s % kStages, use = s / kStages;
+        if (use > 0 && !mbar_wait(smem_addr(&sh.empty[stage]), uint32_t(use - 1) & 1u)) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutEmpty); break; }
+        const int64_t item = first + s / g_count;
+        const int tile = int(item % tiles_per_row), bh = int(item / tiles_per_row);
+        const int hm = bh % p.Hm, b = bh / p.Hm;
+        const int g = ((p.Hm == 1) ? 0 : hm) + s % g_count;
+        const uint32_t dst = stage0 + uint32_t(stage) * kStageBytes, bar = smem_addr(&sh.full[stage]);
+        mbar_arrive_expect_tx(bar, kStageBytes);
+        const int n0 = n_begin + tile * kTileM;
+        tma_load_4d(dst, &map_k, bar, 0, n0, g, b);
+        tma_load_4d(dst + kAHalf, &map_k, bar, 64, n0, g, b);
+        tma_load_2d(dst + 2 * kAHalf, &map_b, bar, 0, g * kNcols);
+        tma_load_2d(dst + 2 * kAHalf + kBHalf, &map_b, bar, 64, g * kNcols);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ================================ MMA issuer ============================================
+    if (lane == 0) {
+      // M = 128, N = 96, fp32 accumulate, bf16 x bf16, both operands K-major
+      constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(kNcols >> 3) << 17) | (uint32_t(kTileM >> 4) << 24);
+      for (int s = 0; s < n_steps; ++s) {
+        const int stage = s % kStages, use = s / kStages, buf = s & 1, acc_use = s >> 1;
+        if (acc_use > 0 && !mbar_wait(smem_addr(&sh.acc_empty[buf]), uint32_t(acc_use - 1) & 1u)) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutEmpty); break; }
+        if (!mbar_wait(smem_addr(&sh.full[stage]), uint32_t(use) & 1u)) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutFull); break; }
+        tc_fence_after();
+        const uint32_t a0 = stage0 + uint32_t(stage) * kStageBytes, b0 = a0 + 2 * kAHalf;
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k) {
+          const uint32_t half = k >> 2, koff = uint32_t(k & 3) * 32u;     // 16 channels = 32 bytes inside the swizzle row
+          umma_bf16(tmem + uint32_t(buf) * 128u, umma_desc(a0 + half * kAHalf + koff), umma_desc(b0 + half * kBHalf + koff),
+                    idesc, k > 0 ? 1u : 0u);
+        }
+        umma_commit(smem_addr(&sh.empty[stage]));         // the stage may be refilled once these MMAs have read it
+        umma_commit(smem_addr(&sh.acc_full[buf]));        // ... and the accumulator is complete
+      }
+    }
+    __syncwarp();
+  } else {
+    // ================================ epilogue ==============================================
+    const int quarter = warp & 3;                          // tensor-memory lanes 32 * quarter .. + 31
+    const int row = quarter * 32 + lane;                   // token row of the tile owned by this thread
+    float acc[kR];
+#pragma unroll
+    for (int j = 0; j < kR; ++j) acc[j] = 0.f;
+    bool ok = true;
+    for (int s = 0; s < n_steps && ok; ++s) {
+      const int buf = s & 1, acc_use = s >> 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.acc_full[buf]), uint32_t(acc_use) & 1u));
+      if (!ok) { if (lane == 0) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutFull); } break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem + (uint32_t(quarter * 32) << 16) + uint32_t(buf) * 128u;
+      float hi[32], mid[32], lo[32];
+      tmem_ld32(taddr, hi);
+      tmem_ld32(taddr + 32, mid);
+      tmem_ld32(taddr + 64, lo);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_addr(&sh.acc_empty[buf]));
+#pragma unroll
+      for (int j = 0; j < kR; ++j) acc[j] += (lo[j] + mid[j]) + hi[j];
+      if ((s + 1) % g_count == 0) {                        // last head of the item: one rounding, one row out
+        const int64_t item = first + s / g_count;
+        const int tile = int(item % tiles_per_row), bh = int(item / tiles_per_row);
+        const int hm = bh % p.Hm, b = bh / p.Hm;
+        const int n = n_begin + tile * kTileM + row;
+        if (n < n_end) {
+          META_T* dst = meta + int64_t(b) * p.meta_sb + int64_t(hm) * p.meta_sh + int64_t(n) * p.meta_sn;
+          if constexpr (sizeof(META_T) == 2) {
+            uint32_t w[kR / 2];
+#pragma unroll
+            for (int j = 0; j < kR / 2; ++j) {
+              const __half2 h = __floats2half2_rn(acc[2 * j], acc[2 * j + 1]);
+              w[j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+#pragma unroll
+            for (int j = 0; j < kR / 8; ++j)
+              reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < kR / 4; ++j)
+              reinterpret_cast<float4*>(dst)[j] = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < kR; ++j) acc[j] = 0.f;
+      }
+    }
+  }
+
+  // ---- teardown: every loop above is bounded, so every warp arrives ------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (sh.abort && threadIdx.x == 0) {
+    // a wait gave up: give copies that may still be in flight a bounded chance to land
+    for (int s = 0; s < kStages; ++s) { mbar_wait(smem_addr(&sh.full[s]), 0); mbar_wait(smem_addr(&sh.full[s]), 1); }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---- host: tensor maps through the driver entry point (no link against libcuda) --------------------------
+using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiled encode_fn() {
+  static EncodeTiled fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiled>(ptr);
+  });
+  return fn;
+}
+
+}  // namespace
+
+size_t project_keys_umma_scratch_bytes(const Problem& p) {
+  if (p.kv_dtype != KVSWAP_BF16 || p.d != kD || p.r != kR) return 0;
+  return size_t(p.Hkv) * kNcols * kD * sizeof(__nv_bfloat16);
+}
+
+// Returns true (and sets *result) when this path took the problem.
+bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
+                                  int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result) {
+  if (scratch == nullptr || project_keys_umma_scratch_bytes(p) == 0) return false;
+  if (p.kv_sn != kD && (p.kv_sn * 2) % 16 != 0) return false;
+  EncodeTiled enc = encode_fn();
+  if (enc == nullptr) return false;
+
+  CUtensorMap map_k, map_b;
+  {
+    const cuuint64_t dims[4] = {cuuint64_t(kD), cuuint64_t(p.N), cuuint64_t(p.Hkv), cuuint64_t(p.B)};
+    const cuuint64_t strides[3] = {cuuint64_t(p.kv_sn) * 2, cuuint64_t(p.kv_sh) * 2, cuuint64_t(p.kv_sb) * 2};
+    const cuuint32_t box[4] = {64, kTileM, 1, 1}, estr[4] = {1, 1, 1, 1};
+    if (enc(&map_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  {
+    const cuuint64_t dims[2] = {cuuint64_t(kD), cuuint64_t(p.Hkv) * kNcols};
+    const cuuint64_t strides[1] = {cuuint64_t(kD) * 2};
+    const cuuint32_t box[2] = {64, kNcols}, estr[2] = {1, 1};
+    if (enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, scratch, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  const int n_proj = p.Hkv * kD * kR;
+  split_adapter_kernel<<<(n_proj + 255) / 256, 256, 0, st>>>(proj, static_cast<__nv_bfloat16*>(scratch), n_proj);
+  *result = cudaGetLastError();
+  if (*result != cudaSuccess) return true;
+
+  const int tiles_per_row = (n_end - n_begin + kTileM - 1) / kTileM;
+  const int64_t items = int64_t(p.B) * p.Hm * tiles_per_row;
+  const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(kNumSMs, items)));
+  const size_t smem = size_t(kStages) * kStageBytes + 1024;
+  auto go = [&](auto kern, auto* meta_t) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (e != cudaSuccess) return e;
+    kern<<<ctas, kThreadsUmma, smem, st>>>(p, map_k, map_b, meta_t, n_begin, n_end, tiles_per_row, err);
+    return cudaGetLastError();
+  };
+  if (p.meta_dtype == KVSWAP_F16) *result = go(project_keys_umma_kernel<__half>, static_cast<__half*>(meta));
+  else *result = go(project_keys_umma_kernel<float>, static_cast<float*>(meta));
+  return true;
+}
+
+}  // namespace kvswap
