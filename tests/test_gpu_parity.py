@@ -283,6 +283,23 @@ def test_project_keys_token_range_leaves_other_rows_untouched():
     np.testing.assert_allclose(got[:, :, 130:517], want[:, :, 130:517], rtol=1e-5, atol=1e-5)
 
 
+def test_project_keys_without_workspace_takes_the_warp_level_path():
+    """kvswap_project_keys accepts ws = NULL: the tcgen05 kernel needs scratch for the split adapter,
+    so the call then runs on the warp-level tensor-core kernel; both must match the oracle."""
+    li = layer(W.CONFIGS[2], 0, 1)
+    wl = li.wl
+    dl = DeviceLayer(li, KV)
+    meta_or = O.project_keys(li.K, li.proj, 1, META_NAME[wl.meta_dtype])
+    tol = project_tolerance(li.K, li.proj, 1, meta_or, wl.meta_dtype)
+    for ws in (dl.ws, None):
+        dl.meta.fill_(float("nan"))
+        kv.kvswap_project_keys(dl.shape, dl.K, dl.proj, dl.meta, 0, wl.n_ctx, ws)
+        torch.cuda.synchronize()
+        got = rt.to_host_f32(dl.meta)
+        assert np.all(np.abs(got.astype(np.float64) - meta_or.astype(np.float64)) <= tol)
+        assert np.mean(got != meta_or.astype(np.float32)) < 0.02
+
+
 def test_strided_kv_and_metadata_views():
     """K and V interleaved in one buffer (row stride 2d) and metadata rows padded."""
     wl = small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, n_ctx=517, group_size=8)
