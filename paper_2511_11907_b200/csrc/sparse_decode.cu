@@ -237,7 +237,7 @@ struct AluEngine {
     }
   }
 
-  // sm_m, sm_l: [4] per warp;  sm_acc: [RH][D] per warp
+  // sm_m, sm_l: [8] per warp;  sm_acc: [RH][D] per warp
   __device__ __forceinline__ void store(float* sm_m, float* sm_l, float* sm_acc) const {
     if (lane < 4) { sm_m[lane] = m_run; sm_l[lane] = l_run; }
 #pragma unroll
@@ -382,7 +382,7 @@ struct MmaEngine {
   }
 
   __device__ __forceinline__ void store(float* sm_m, float* sm_l, float* sm_acc) const {
-    if (t == 0 && g < 4) { sm_m[g] = m_run; sm_l[g] = l_run; }
+    if (t == 0) { sm_m[g] = m_run; sm_l[g] = l_run; }        // g = 0..7: one slot per possible head
 #pragma unroll
     for (int i = 0; i < KS; ++i)
 #pragma unroll
@@ -533,22 +533,22 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   // ---- merge the warps of the CTA ------------------------------------------------------------------
   __syncthreads();
   // The ring is idle now (every copy was waited for); reuse it for the merge.
-  float* sm_m = reinterpret_cast<float*>(ring_ptr);                 // [kWarps][4]
-  float* sm_l = sm_m + kWarps * 4;                                  // [kWarps][4]
-  float* sm_acc = sm_l + kWarps * 4;                                // [kWarps][RH][D]
-  eng.store(sm_m + warp * 4, sm_l + warp * 4, sm_acc + warp * RH * D);
+  float* sm_m = reinterpret_cast<float*>(ring_ptr);                 // [kWarps][8]
+  float* sm_l = sm_m + kWarps * 8;                                  // [kWarps][8]
+  float* sm_acc = sm_l + kWarps * 8;                                // [kWarps][RH][D]
+  eng.store(sm_m + warp * 8, sm_l + warp * 8, sm_acc + warp * RH * D);
   __syncthreads();
   for (int i = threadIdx.x; i < RH * D; i += kThreads) {
     const int hh = i / D, c = i % D;
     float mx = -INFINITY;
 #pragma unroll
-    for (int k = 0; k < kWarps; ++k) mx = fmaxf(mx, sm_m[k * 4 + hh]);
+    for (int k = 0; k < kWarps; ++k) mx = fmaxf(mx, sm_m[k * 8 + hh]);
     float lsum = 0.f, a = 0.f;
     if (mx > -INFINITY) {
 #pragma unroll
       for (int k = 0; k < kWarps; ++k) {
-        const float w = ex2(sm_m[k * 4 + hh] - mx);
-        lsum = fmaf(sm_l[k * 4 + hh], w, lsum);
+        const float w = ex2(sm_m[k * 8 + hh] - mx);
+        lsum = fmaf(sm_l[k * 8 + hh], w, lsum);
         a = fmaf(sm_acc[(k * RH + hh) * D + c], w, a);
       }
     }
@@ -616,9 +616,11 @@ cudaError_t launch_one(const Problem& p, const Workspace& w, const void* q, cons
   const size_t smem = kControlBytes + 128 + size_t(kWarps) * depth * stage_bytes<KV_T, D>();
   int g_shift = -1;
   for (int sft = 0; sft < 31; ++sft) if ((1 << sft) == p.G) g_shift = sft;
-  // Tensor-core engine for 16-bit K/V with q of the same type and at least two heads per K/V row.
-  constexpr bool kMma = sizeof(KV_T) == 2 && std::is_same<KV_T, Q_T>::value && RH >= 2;
-  using Engine = typename std::conditional<kMma, MmaEngine<KV_T, KV_T, D, RH>, AluEngine<KV_T, Q_T, D, RH>>::type;
+  // Tensor-core engine for 16-bit K/V with q of the same type (up to 8 heads per K/V row); the
+  // fp32-pipe engine otherwise (up to 4).
+  constexpr bool kMma = sizeof(KV_T) == 2 && std::is_same<KV_T, Q_T>::value;
+  using Engine = typename std::conditional<kMma, MmaEngine<KV_T, KV_T, D, RH>, AluEngine<KV_T, Q_T, D, (RH <= 4 ? RH : 4)>>::type;
+  if (!kMma && RH > 4) return cudaErrorInvalidValue;             // never planned: see plan_sparse_decode
   auto kern = sparse_decode_splitk_kernel<KV_T, Q_T, D, RH, Engine>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
   if (e != cudaSuccess) return e;
@@ -635,6 +637,10 @@ cudaError_t launch_rh(const Problem& p, const Workspace& w, const void* q, const
                       const int32_t* gi, const int32_t* ns, float* partial, float* out, float* lse, uint32_t* err,
                       cudaStream_t st) {
   switch (w.heads_per_cta) {
+    case 8: return launch_one<KV_T, Q_T, D, 8>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
+    case 7: return launch_one<KV_T, Q_T, D, 7>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
+    case 6: return launch_one<KV_T, Q_T, D, 6>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
+    case 5: return launch_one<KV_T, Q_T, D, 5>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
     case 4: return launch_one<KV_T, Q_T, D, 4>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
     case 3: return launch_one<KV_T, Q_T, D, 3>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
     case 2: return launch_one<KV_T, Q_T, D, 2>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
@@ -665,7 +671,9 @@ cudaError_t launch_q(const Problem& p, const Workspace& w, const void* q, const 
 void plan_sparse_decode(const Problem& p, Workspace* w) {
   // rho query heads share each K/V row; a CTA serves up to 4 of them per pass.
   int rh = 1;
-  for (int c = 4; c >= 1; --c) if (p.rho % c == 0) { rh = c; break; }
+  // the tensor-core engine (16-bit K/V, q of the same type) takes up to 8, the fp32-pipe engine up to 4
+  const int rh_max = (p.kv_dtype != KVSWAP_F32 && p.q_dtype == p.kv_dtype) ? 8 : 4;
+  for (int c = rh_max; c >= 1; --c) if (p.rho % c == 0) { rh = c; break; }
   w->heads_per_cta = rh;
   const int64_t problems = int64_t(p.B) * p.Hkv * (p.rho / rh);
   const int64_t tokens = int64_t(p.M) * p.G + (p.N - int64_t(p.NG) * p.G);

@@ -184,6 +184,14 @@ EDGE = {
                             n_q_heads=6, n_kv_heads=2, n_ctx=8 * 90 + 3, top_k=12),
     "bf16_rank_64": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=64, group_size=8,
                           n_ctx=8 * 64 + 1, top_k=10),
+    "bf16_gqa_ratio_8": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=8,
+                              n_q_heads=16, n_kv_heads=2, n_ctx=8 * 70 + 5, top_k=14),
+    "bf16_gqa_ratio_5": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=64, rank=32, group_size=4,
+                              n_q_heads=10, n_kv_heads=2, n_ctx=4 * 130 + 1, top_k=21),
+    "fp16_gqa_ratio_6": small(kv_dtype=W.F16, q_dtype=W.F16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=8,
+                              n_q_heads=12, n_kv_heads=2, n_ctx=8 * 60, top_k=9),
+    "bf16_gqa_ratio_1": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=8,
+                              n_q_heads=2, n_kv_heads=2, n_ctx=8 * 50 + 3, top_k=8),
     # long score rows: 16 keys per thread in the register top-k, and the shared-memory top-k beyond it
     "ten_thousand_groups": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=64, rank=32,
                                  group_size=4, batch=1, n_ctx=4 * 10000 + 3, top_k=700),
