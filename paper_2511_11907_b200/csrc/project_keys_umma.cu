@@ -18,13 +18,11 @@
 //   warps 2-5 epilogue: tcgen05.ld of the finished accumulator (one token row per thread), sum of
 //            the three pieces, running sum over heads, one rounding into the metadata type.
 // Stages and accumulators are handed over through mbarriers; every wait is bounded.
-#include <cuda.h>
-
 #include <algorithm>
-#include <mutex>
 
 #include "async_copy.cuh"
 #include "common.cuh"
+#include "tensor_map.cuh"
 
 namespace kvswap {
 namespace {
@@ -53,15 +51,6 @@ __global__ void split_adapter_kernel(const float* __restrict__ proj, __nv_bfloat
 }
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
-  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
 // K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_byte_addr) {
   return uint64_t((smem_byte_addr >> 4) & 0x3fffu) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) |
@@ -242,24 +231,6 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
   }
 }
 
-// ---- host: tensor maps through the driver entry point (no link against libcuda) --------------------------
-using EncodeTiled = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiled encode_fn() {
-  static EncodeTiled fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiled>(ptr);
-  });
-  return fn;
-}
-
 }  // namespace
 
 size_t project_keys_umma_scratch_bytes(const Problem& p) {
@@ -272,19 +243,10 @@ bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* 
                                   int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result) {
   if (scratch == nullptr || project_keys_umma_scratch_bytes(p) == 0) return false;
   if (p.kv_sn != kD && (p.kv_sn * 2) % 16 != 0) return false;
-  EncodeTiled enc = encode_fn();
+  EncodeTiledFn enc = tensor_map_encoder();
   if (enc == nullptr) return false;
-
   CUtensorMap map_k, map_b;
-  {
-    const cuuint64_t dims[4] = {cuuint64_t(kD), cuuint64_t(p.N), cuuint64_t(p.Hkv), cuuint64_t(p.B)};
-    const cuuint64_t strides[3] = {cuuint64_t(p.kv_sn) * 2, cuuint64_t(p.kv_sh) * 2, cuuint64_t(p.kv_sb) * 2};
-    const cuuint32_t box[4] = {64, kTileM, 1, 1}, estr[4] = {1, 1, 1, 1};
-    if (enc(&map_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return false;
-  }
+  if (!make_rows_tensor_map(&map_k, K, 2, true, kD, p.N, p.Hkv, p.B, p.kv_sn, p.kv_sh, p.kv_sb, kTileM)) return false;
   {
     const cuuint64_t dims[2] = {cuuint64_t(kD), cuuint64_t(p.Hkv) * kNcols};
     const cuuint64_t strides[1] = {cuuint64_t(kD) * 2};
