@@ -670,15 +670,18 @@ cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, flo
   const bool streaming = one_term && g_shift >= 0 && p.r * int(sizeof(META_T)) == kRowBytes && p.meta_sn == p.r &&
                          tile_items < (int64_t(1) << 30);
   if (streaming) {
-    const int ns = (p.Hm == 1) ? p.S : 1;
     // fp16 metadata: the tensor-core scorer serves every streaming case (with one score per
     // row it uses one of its eight columns; it is still far cheaper in instructions per row
     // than the fp32 pipes, which at one dot product per 64-byte row are issue-bound, not HBM-bound).
-    if constexpr (std::is_same<META_T, __half>::value) return launch_mma(p, uq, meta, scores, g_shift, err, st);
-    if (ns == 1) return launch_tiles<META_T, 1>(p, uq, meta, scores, g_shift, err, st);
-    if (ns == 2) return launch_tiles<META_T, 2>(p, uq, meta, scores, g_shift, err, st);
-    if (ns <= 4) return launch_tiles<META_T, 4>(p, uq, meta, scores, g_shift, err, st);
-    return launch_tiles<META_T, 8>(p, uq, meta, scores, g_shift, err, st);
+    if constexpr (std::is_same<META_T, __half>::value) {
+      return launch_mma(p, uq, meta, scores, g_shift, err, st);
+    } else {
+      const int ns = (p.Hm == 1) ? p.S : 1;
+      if (ns == 1) return launch_tiles<META_T, 1>(p, uq, meta, scores, g_shift, err, st);
+      if (ns == 2) return launch_tiles<META_T, 2>(p, uq, meta, scores, g_shift, err, st);
+      if (ns <= 4) return launch_tiles<META_T, 4>(p, uq, meta, scores, g_shift, err, st);
+      return launch_tiles<META_T, 8>(p, uq, meta, scores, g_shift, err, st);
+    }
   }
   if (p.Hm == 1) {
     if (p.S == 1) return launch_ns<META_T, 1>(p, uq, meta, scores, 1, st);
