@@ -217,6 +217,9 @@ typedef struct {
  *   group_idx  [L, B, S, M] int32, n_selected [L, B, S] int32: the selections of this step, kept
  *              per layer so that the caller can compare consecutive steps (Sec. 4.4.2).
  * `ws` is shared by all layers (size: kvswap_workspace_bytes).  probe_opt may be NULL.
+ * Because all L queries are given at once, the low-rank queries Q A of Eq. 1 are computed for
+ * many layers by one launch ahead of the per-layer work; results are identical to calling
+ * kvswap_score_select and kvswap_sparse_decode layer by layer.
  */
 int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q,
                        float* out, float* lse_opt, int32_t* group_idx, int32_t* n_selected,

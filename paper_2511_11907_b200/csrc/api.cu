@@ -63,7 +63,10 @@ void plan_workspace(const Problem& p, Workspace* w) {
   plan_sparse_decode(p, w);
 
   size_t off = 256;  // first 256 bytes reserved
-  w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
+  // Room for the low-rank queries of several layers (at most 1 MiB beyond one layer's worth).
+  const size_t uq_layer = sizeof(float) * size_t(p.B) * p.Su * p.r;
+  w->uq_layers = int(std::min<size_t>(kMaxQueryLayers, std::max<size_t>(1, (size_t(1) << 20) / uq_layer)));
+  w->off_uq = off;       off += align256(uq_layer * w->uq_layers);
   w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * std::max(p.NG, 1));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
   w->off_adapter = off;  off += align256(project_keys_umma_scratch_bytes(p) + 1024);   // 1 KiB: tensor-map base alignment
@@ -118,11 +121,11 @@ int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* p
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 
-int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
-                        int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
-                        size_t ws_bytes, void* cuda_stream) {
-  Problem p;
-  int st = resolve(shape, &p);
+// Argument checks of kvswap_score_select; fills the problem and the workspace plan.
+static int check_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
+                              const int32_t* group_idx, const int32_t* n_selected, const float* group_scores_opt,
+                              const void* ws, size_t ws_bytes, Problem* p, Workspace* w) {
+  int st = resolve(shape, p);
   if (st != KVSWAP_OK) return st;
   if (q == nullptr || proj == nullptr || meta == nullptr || group_idx == nullptr || n_selected == nullptr ||
       ws == nullptr)
@@ -131,17 +134,33 @@ int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* p
       (reinterpret_cast<uintptr_t>(group_idx) & 3u) || (reinterpret_cast<uintptr_t>(n_selected) & 3u) ||
       (group_scores_opt && misaligned(group_scores_opt)))
     return KVSWAP_ERR_ALIGN;
-  Workspace w;
-  plan_workspace(p, &w);
-  if (ws_bytes < w.total) return KVSWAP_ERR_WORKSPACE;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  char* base = static_cast<char*>(ws);
-  float* uq = reinterpret_cast<float*>(base + w.off_uq);
-  float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
+  plan_workspace(*p, w);
+  if (ws_bytes < w->total) return KVSWAP_ERR_WORKSPACE;
+  return KVSWAP_OK;
+}
 
-  cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
-  if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
+// Scoring, pooling and selection of one layer from low-rank queries `uq` that are already in place.
+static cudaError_t score_select_from_uq(const Problem& p, const Workspace& w, const float* uq, const void* meta,
+                                        int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
+                                        cudaStream_t stream) {
+  float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_scores);
+  cudaError_t e = cudaSuccess;
+  if (p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
   if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
+  return e;
+}
+
+int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
+                        int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
+                        size_t ws_bytes, void* cuda_stream) {
+  Problem p;
+  Workspace w;
+  int st = check_score_select(shape, q, proj, meta, group_idx, n_selected, group_scores_opt, ws, ws_bytes, &p, &w);
+  if (st != KVSWAP_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  float* uq = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_uq);
+  cudaError_t e = launch_lowrank_query_layers(p, q, &proj, 1, uq, stream);
+  if (e == cudaSuccess) e = score_select_from_uq(p, w, uq, meta, group_idx, n_selected, group_scores_opt, ws, stream);
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 
@@ -188,20 +207,38 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
   const size_t q_bytes = size_t(p.B) * p.Hq * p.d * dtype_bytes(p.q_dtype);
   const size_t out_elems = size_t(p.B) * p.Hq * p.d;
   const size_t idx_elems = size_t(p.B) * p.S * p.M, nsel_elems = size_t(p.B) * p.S;
-  for (int l = 0; l < layers->n_layers; ++l) {
-    const bool probed = probe_opt != nullptr && probe_opt->layer == l;
-    const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-    int32_t* idx_l = group_idx + size_t(l) * idx_elems;
-    int32_t* nsel_l = n_selected + size_t(l) * nsel_elems;
-    if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), stream);
-    st = kvswap_score_select(shape, ql, layers->proj[l], layers->meta[l], idx_l, nsel_l, nullptr, ws, ws_bytes,
-                             cuda_stream);
-    if (st != KVSWAP_OK) return st;
-    if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), stream);
-    st = kvswap_sparse_decode(shape, ql, layers->K[l], layers->V[l], idx_l, nsel_l, out + size_t(l) * out_elems,
-                              lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes, cuda_stream);
-    if (st != KVSWAP_OK) return st;
-    if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
+  // The step is handed the queries of every layer, so their low-rank projections (Eq. 1's Q A) are
+  // taken off each layer's critical path: one launch computes them for as many layers as the
+  // workspace holds, and each layer then runs scoring, selection and attention only.
+  Workspace w;
+  st = check_score_select(shape, q, layers->proj[0], layers->meta[0], group_idx, n_selected, nullptr, ws, ws_bytes,
+                          &p, &w);
+  if (st != KVSWAP_OK) return st;
+  for (int l0 = 0; l0 < layers->n_layers; l0 += w.uq_layers) {
+    const void* q0 = static_cast<const char*>(q) + size_t(l0) * q_bytes;
+    const int n_ahead = std::min(w.uq_layers, layers->n_layers - l0);
+    for (int l = l0; l < l0 + n_ahead; ++l) {
+      if (layers->proj[l] == nullptr || layers->meta[l] == nullptr) return KVSWAP_ERR_NULL;
+      if (misaligned(layers->proj[l]) || misaligned(layers->meta[l])) return KVSWAP_ERR_ALIGN;
+    }
+    float* uq0 = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_uq);
+    if (launch_lowrank_query_layers(p, q0, layers->proj + l0, n_ahead, uq0, stream) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+    for (int l = l0; l < l0 + n_ahead; ++l) {
+      const bool probed = probe_opt != nullptr && probe_opt->layer == l;
+      const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+      int32_t* idx_l = group_idx + size_t(l) * idx_elems;
+      int32_t* nsel_l = n_selected + size_t(l) * nsel_elems;
+      if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), stream);
+      const float* uq = uq0 + size_t(l - l0) * p.B * p.Su * p.r;
+      if (score_select_from_uq(p, w, uq, layers->meta[l], idx_l, nsel_l, nullptr, ws, stream) != cudaSuccess)
+        return KVSWAP_ERR_CUDA;
+      if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), stream);
+      st = kvswap_sparse_decode(shape, ql, layers->K[l], layers->V[l], idx_l, nsel_l, out + size_t(l) * out_elems,
+                                lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes, cuda_stream);
+      if (st != KVSWAP_OK) return st;
+      if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
+    }
   }
   return KVSWAP_OK;
 }

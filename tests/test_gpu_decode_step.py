@@ -1,0 +1,83 @@
+"""kvswap_decode_step (all layers of one decode step in one call, low-rank queries computed for
+many layers ahead of the per-layer work) gives exactly what the three per-layer calls give.
+The per-layer calls themselves are checked against the oracle in test_gpu_parity.py."""
+import pytest
+import torch
+
+from paper_2511_11907_b200 import binding as kv
+from paper_2511_11907_b200 import device_workload as DW
+from paper_2511_11907_b200 import runtime as rt
+from paper_2511_11907_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _step_buffers(dw):
+    wl, s = dw.wl, dw.shape
+    L, B = wl.layers, wl.batch
+    out = torch.full((L, B, wl.n_q_heads, wl.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+    lse = torch.full((L, B, wl.n_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    idx = torch.full((L, B, s.n_scopes, wl.top_k), -7, dtype=torch.int32, device="cuda")
+    nsel = torch.full((L, B, s.n_scopes), -7, dtype=torch.int32, device="cuda")
+    return out, lse, idx, nsel
+
+
+def _run_case(wl, meta_heads, scope):
+    dw = DW.build(wl, 1 if meta_heads == "joint" else wl.n_kv_heads, scope, walk_steps=1, reserve_bytes=1 << 30)
+    assert dw.layers_resident == wl.layers
+    ws = rt.alloc_workspace(dw.shape)
+    for l in range(wl.layers):
+        kv.kvswap_project_keys(dw.shape, dw.K[l], dw.proj[l], dw.meta[l], 0, wl.n_ctx, ws)
+    q = dw.q_walk[0]
+
+    # layer by layer through the three public calls
+    out_a, lse_a, idx_a, nsel_a = _step_buffers(dw)
+    for l in range(wl.layers):
+        kv.kvswap_score_select(dw.shape, q[l], dw.proj[l], dw.meta[l], idx_a[l], nsel_a[l], None, ws)
+        kv.kvswap_sparse_decode(dw.shape, q[l], dw.K[l], dw.V[l], idx_a[l], nsel_a[l], out_a[l], lse_a[l], ws)
+    torch.cuda.synchronize()
+    assert kv.kvswap_read_device_status(ws) == 0
+
+    # the whole step in one call
+    ws.fill_(0xFF)
+    kv.kvswap_workspace_init(ws)
+    out_b, lse_b, idx_b, nsel_b = _step_buffers(dw)
+    kv.kvswap_decode_step(dw.shape, dw.layer_tables(), q, out_b, lse_b, idx_b, nsel_b, ws)
+    torch.cuda.synchronize()
+    assert kv.kvswap_read_device_status(ws) == 0
+    assert torch.equal(nsel_a, nsel_b)
+    assert torch.equal(idx_a, idx_b)
+    assert not torch.isnan(out_b).any()
+    assert torch.equal(out_a, out_b)
+    assert torch.equal(lse_a, lse_b)
+
+    # the same step with queries and outputs in host memory
+    out_c, _, idx_c, nsel_c = _step_buffers(dw)
+    q_host = q.cpu().pin_memory()
+    out_host = torch.full(out_c.shape, float("nan"), dtype=torch.float32).pin_memory()
+    q_dev = torch.zeros_like(q)
+    kv.kvswap_decode_step_host(dw.shape, dw.layer_tables(), q_host, out_host, q_dev, out_c, idx_c, nsel_c, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(idx_a, idx_c)
+    assert torch.equal(out_a.cpu(), out_host)
+
+
+@pytest.mark.parametrize("meta_heads", ["joint", "per_head"])
+@pytest.mark.parametrize("scope", [W.SCOPE_KV_HEAD, W.SCOPE_ALL_HEADS])
+def test_decode_step_equals_layer_by_layer_calls(meta_heads, scope):
+    wl = W.CONFIGS[4].reduced("cfg4-step", layers=5, batch=2, n_ctx=4096 + 11, top_k=24, calib_rows=1024)
+    _run_case(wl, meta_heads, scope)
+
+
+def test_decode_step_with_more_layers_than_one_query_launch_serves():
+    """70 layers: the low-rank queries are computed in two launches (64 layers, then 6)."""
+    wl = W.CONFIGS[3].reduced("cfg3-deep", layers=70, batch=1, n_ctx=1024 + 3, top_k=16, calib_rows=1024,
+                              n_q_heads=8, n_kv_heads=2)
+    _run_case(wl, "joint", W.SCOPE_KV_HEAD)
+
+
+def test_decode_step_when_the_workspace_holds_few_layers_of_queries():
+    """fp32, large batch x rank: one layer's low-rank queries take 256 KiB, so four layers go per launch."""
+    wl = W.CONFIGS[1].reduced("cfg1-wide", layers=6, batch=64, n_ctx=512, rank=128, head_dim=128, n_q_heads=32,
+                              n_kv_heads=8, top_k=8, calib_rows=1536)
+    _run_case(wl, "per_head", W.SCOPE_KV_HEAD)
