@@ -286,6 +286,21 @@ def run_ours(args, wl):
     select_ms = [p[0].elapsed_time(p[1]) for p in probes]
     decode_ms = [p[1].elapsed_time(p[2]) for p in probes]
 
+    # ---- the same step with the predictor held to one layer ahead of the attention (what a model's
+    # own layer-to-layer dependency allows); reported beside the headline, which uses the default --------
+    layers_1 = dw.layer_tables(max_lookahead=1)
+    n1 = max(1, min(steps, 100))
+    for i in range(3):
+        kv.kvswap_decode_step(shape, layers_1, dw.q_walk[i % n_walk], out, None, idx, nsel, ws, None)
+    a1, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    a1.record()
+    for i in range(n1):
+        kv.kvswap_decode_step(shape, layers_1, dw.q_walk[i % n_walk], out, None, idx, nsel, ws, None)
+    b1.record()
+    sync_all()
+    look1_ms = a1.elapsed_time(b1)
+
     # ---- each call on its own, back to back over all layers (every launch reads a different layer's
     # buffers, so nothing is served from L2): the average launch duration the roofline uses -----------
     def per_call_ms(fn):
@@ -343,7 +358,7 @@ def run_ours(args, wl):
     clocks = sampler.stop(wall0, wall1) if sampler else None
 
     # ---- max over ranks ----------------------------------------------------------------------------
-    elapsed_ms, e2e_ms = shard.max_over_ranks([elapsed_ms, e2e_ms], device=dev)
+    elapsed_ms, e2e_ms, look1_ms = shard.max_over_ranks([elapsed_ms, e2e_ms, look1_ms], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -375,6 +390,9 @@ def run_ours(args, wl):
                          f"{dw.layers_resident} distinct KV stores (>> 126 MB) before any buffer repeats",
                    "kv_resident_gb": round(dw.layers_resident * 2 * dw.K[0].numel() * esz[wl.kv_dtype] / 1e9, 1)},
         "keys_scored_per_sec": value * keys_per_step,
+        "schedule": {"predictor_lookahead_layers": 3,
+                     "lookahead_1": {"value": world * 1e3 * n1 / look1_ms, "unit": UNIT, "steps": n1,
+                                     "ms_per_step": look1_ms / n1}},
         "e2e": {"value": world * 1e3 * e2e_steps / e2e_ms, "unit": UNIT, "h2d_bytes_per_step": q_bytes,
                 "d2h_bytes_per_step": out_bytes, "steps": e2e_steps},
         "gpu_launches": 5 * L * steps,

@@ -185,10 +185,14 @@ int kvswap_sparse_decode_static(const kvswap_shape* shape, const void* q, const 
 /*
  * Per-layer tensors of a model with L layers that all share one kvswap_shape.  Each member is a
  * HOST array of L DEVICE pointers: K[l], V[l] are [B, H_kv, N, d]; meta[l] is [B, H_m, N, r];
- * proj[l] is [H_kv, d, r] fp32.
+ * proj[l] is [H_kv, d, r] fp32.  max_lookahead bounds how many layers kvswap_decode_step's
+ * predictor may run ahead of its attention: 1 = layer l is predicted while layer l-1 is attended
+ * (what a model allows, whose layer-l prediction needs the input of layer l-1); 0 = the
+ * library's default (3).  Negative values are KVSWAP_ERR_SHAPE.
  */
 typedef struct {
   int32_t n_layers;
+  int32_t max_lookahead;
   const void* const* K;
   const void* const* V;
   const void* const* meta;
@@ -217,9 +221,16 @@ typedef struct {
  *   group_idx  [L, B, S, M] int32, n_selected [L, B, S] int32: the selections of this step, kept
  *              per layer so that the caller can compare consecutive steps (Sec. 4.4.2).
  * `ws` is shared by all layers (size: kvswap_workspace_bytes).  probe_opt may be NULL.
- * Because all L queries are given at once, the low-rank queries Q A of Eq. 1 are computed for
- * many layers by one launch ahead of the per-layer work; results are identical to calling
- * kvswap_score_select and kvswap_sparse_decode layer by layer.
+ * The call overlaps prediction and attention as the paper's runtime does (Sec. 4.3 "Online
+ * prediction", Sec. 4.4): the predictor (kvswap_score_select's kernels) runs on an internal
+ * stream, at most layers->max_lookahead layers ahead of the attention (kvswap_sparse_decode's
+ * kernels) on `cuda_stream`; all L queries being given, no data dependency forbids it.  The
+ * internal stream is ordered after the work already in `cuda_stream` and has joined it again
+ * when the step's last kernel is in it, so the caller synchronises `cuda_stream` only.  The
+ * internal stream and its events are created on a device's first call (later calls allocate
+ * nothing) and calls are serialised by a process-wide lock.  Results are identical to calling
+ * kvswap_score_select and kvswap_sparse_decode layer by layer.  A probe's ev_begin and ev_mid
+ * are recorded on the internal stream, ev_end on `cuda_stream`.
  */
 int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q,
                        float* out, float* lse_opt, int32_t* group_idx, int32_t* n_selected,

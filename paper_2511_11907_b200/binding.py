@@ -148,7 +148,8 @@ def kvswap_version() -> int:
 # Whole decode step over L layers
 # ------------------------------------------------------------------------------------------------
 class kvswap_layers(ctypes.Structure):
-    _fields_ = [("n_layers", ctypes.c_int32), ("K", ctypes.POINTER(ctypes.c_void_p)),
+    _fields_ = [("n_layers", ctypes.c_int32), ("max_lookahead", ctypes.c_int32),
+                ("K", ctypes.POINTER(ctypes.c_void_p)),
                 ("V", ctypes.POINTER(ctypes.c_void_p)), ("meta", ctypes.POINTER(ctypes.c_void_p)),
                 ("proj", ctypes.POINTER(ctypes.c_void_p))]
 
@@ -158,9 +159,10 @@ class kvswap_probe(ctypes.Structure):
                 ("ev_end", ctypes.c_void_p)]
 
 
-def make_layers(K, V, meta, proj) -> kvswap_layers:
+def make_layers(K, V, meta, proj, max_lookahead: int = 0) -> kvswap_layers:
     """Pointer tables for lists of per-layer device tensors.  The returned struct keeps the
-    tensors and the tables alive."""
+    tensors and the tables alive.  max_lookahead: layers the predictor of kvswap_decode_step may
+    run ahead of the attention (0 = library default, 1 = one layer, as a model allows)."""
     n = len(K)
     assert len(V) == n and len(meta) == n and len(proj) == n
 
@@ -168,7 +170,7 @@ def make_layers(K, V, meta, proj) -> kvswap_layers:
         return (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
 
     tabs = [table(K), table(V), table(meta), table(proj)]
-    layers = kvswap_layers(n, *[ctypes.cast(t, ctypes.POINTER(ctypes.c_void_p)) for t in tabs])
+    layers = kvswap_layers(n, int(max_lookahead), *[ctypes.cast(t, ctypes.POINTER(ctypes.c_void_p)) for t in tabs])
     layers._keep = (tabs, list(K), list(V), list(meta), list(proj))
     return layers
 

@@ -2,6 +2,8 @@
 // kernel sequencing.  No entry point allocates or keeps state; only kvswap_read_device_status
 // synchronises.
 #include <algorithm>
+#include <mutex>
+#include <vector>
 
 #include "common.cuh"
 
@@ -63,10 +65,7 @@ void plan_workspace(const Problem& p, Workspace* w) {
   plan_sparse_decode(p, w);
 
   size_t off = 256;  // first 256 bytes reserved
-  // Room for the low-rank queries of several layers (at most 1 MiB beyond one layer's worth).
-  const size_t uq_layer = sizeof(float) * size_t(p.B) * p.Su * p.r;
-  w->uq_layers = int(std::min<size_t>(kMaxQueryLayers, std::max<size_t>(1, (size_t(1) << 20) / uq_layer)));
-  w->off_uq = off;       off += align256(uq_layer * w->uq_layers);
+  w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
   w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * std::max(p.NG, 1));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
   w->off_adapter = off;  off += align256(project_keys_umma_scratch_bytes(p) + 1024);   // 1 KiB: tensor-map base alignment
@@ -139,13 +138,15 @@ static int check_score_select(const kvswap_shape* shape, const void* q, const fl
   return KVSWAP_OK;
 }
 
-// Scoring, pooling and selection of one layer from low-rank queries `uq` that are already in place.
-static cudaError_t score_select_from_uq(const Problem& p, const Workspace& w, const float* uq, const void* meta,
-                                        int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
-                                        cudaStream_t stream) {
-  float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_scores);
-  cudaError_t e = cudaSuccess;
-  if (p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
+// The three launches of the predictor for one layer (arguments already checked).
+static cudaError_t score_select_launch(const Problem& p, const Workspace& w, const void* q, const float* proj,
+                                       const void* meta, int32_t* group_idx, int32_t* n_selected,
+                                       float* group_scores_opt, void* ws, cudaStream_t stream) {
+  char* base = static_cast<char*>(ws);
+  float* uq = reinterpret_cast<float*>(base + w.off_uq);
+  float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
+  cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
+  if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
   if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
   return e;
 }
@@ -157,10 +158,8 @@ int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* p
   Workspace w;
   int st = check_score_select(shape, q, proj, meta, group_idx, n_selected, group_scores_opt, ws, ws_bytes, &p, &w);
   if (st != KVSWAP_OK) return st;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  float* uq = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_uq);
-  cudaError_t e = launch_lowrank_query_layers(p, q, &proj, 1, uq, stream);
-  if (e == cudaSuccess) e = score_select_from_uq(p, w, uq, meta, group_idx, n_selected, group_scores_opt, ws, stream);
+  cudaError_t e = score_select_launch(p, w, q, proj, meta, group_idx, n_selected, group_scores_opt, ws,
+                                      static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 
@@ -190,9 +189,56 @@ static int check_layers(const kvswap_layers* layers) {
   if (layers == nullptr || layers->K == nullptr || layers->V == nullptr || layers->meta == nullptr ||
       layers->proj == nullptr)
     return KVSWAP_ERR_NULL;
-  if (layers->n_layers < 1) return KVSWAP_ERR_SHAPE;
+  if (layers->n_layers < 1 || layers->max_lookahead < 0) return KVSWAP_ERR_SHAPE;
   return KVSWAP_OK;
 }
+
+// Per-device resources of kvswap_decode_step's two-stream schedule: a stream for the predictor and
+// two events per layer.  Created on first use, kept for the life of the process.
+namespace {
+struct StepResources {
+  cudaStream_t predictor = nullptr;
+  cudaEvent_t fork = nullptr;
+  std::vector<cudaEvent_t> selected;     // selected[l]: layer l's selection is written
+  std::vector<cudaEvent_t> attended;     // attended[l]: layer l's attention output is written
+};
+constexpr int kMaxDevices = 64;
+constexpr int kDefaultLookahead = 3;   // layers the predictor may run ahead when the caller sets no limit
+constexpr int kHostLead = 3;           // layers by which the host enqueues the predictor ahead of the attention
+std::mutex g_step_mutex;
+StepResources g_step[kMaxDevices];
+
+cudaError_t grow(std::vector<cudaEvent_t>* evs, int n) {
+  while (int(evs->size()) < n) {
+    cudaEvent_t ev = nullptr;
+    cudaError_t e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) return e;
+    evs->push_back(ev);
+  }
+  return cudaSuccess;
+}
+
+// Must be called with g_step_mutex held.
+cudaError_t step_resources(int n_layers, StepResources** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  StepResources& r = g_step[dev];
+  if (r.predictor == nullptr) {
+    e = cudaStreamCreateWithFlags(&r.predictor, cudaStreamNonBlocking);
+    if (e != cudaSuccess) { r.predictor = nullptr; return e; }
+  }
+  if (r.fork == nullptr) {
+    e = cudaEventCreateWithFlags(&r.fork, cudaEventDisableTiming);
+    if (e != cudaSuccess) { r.fork = nullptr; return e; }
+  }
+  if ((e = grow(&r.selected, n_layers)) != cudaSuccess) return e;
+  if ((e = grow(&r.attended, n_layers)) != cudaSuccess) return e;
+  *out = &r;
+  return cudaSuccess;
+}
+}  // namespace
 
 int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q, float* out,
                        float* lse_opt, int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
@@ -204,43 +250,79 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
   if (st != KVSWAP_OK) return st;
   if (q == nullptr || out == nullptr || group_idx == nullptr || n_selected == nullptr) return KVSWAP_ERR_NULL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int L = layers->n_layers;
   const size_t q_bytes = size_t(p.B) * p.Hq * p.d * dtype_bytes(p.q_dtype);
   const size_t out_elems = size_t(p.B) * p.Hq * p.d;
   const size_t idx_elems = size_t(p.B) * p.S * p.M, nsel_elems = size_t(p.B) * p.S;
-  // The step is handed the queries of every layer, so their low-rank projections (Eq. 1's Q A) are
-  // taken off each layer's critical path: one launch computes them for as many layers as the
-  // workspace holds, and each layer then runs scoring, selection and attention only.
   Workspace w;
   st = check_score_select(shape, q, layers->proj[0], layers->meta[0], group_idx, n_selected, nullptr, ws, ws_bytes,
                           &p, &w);
   if (st != KVSWAP_OK) return st;
-  for (int l0 = 0; l0 < layers->n_layers; l0 += w.uq_layers) {
-    const void* q0 = static_cast<const char*>(q) + size_t(l0) * q_bytes;
-    const int n_ahead = std::min(w.uq_layers, layers->n_layers - l0);
-    for (int l = l0; l < l0 + n_ahead; ++l) {
-      if (layers->proj[l] == nullptr || layers->meta[l] == nullptr) return KVSWAP_ERR_NULL;
-      if (misaligned(layers->proj[l]) || misaligned(layers->meta[l])) return KVSWAP_ERR_ALIGN;
-    }
-    float* uq0 = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_uq);
-    if (launch_lowrank_query_layers(p, q0, layers->proj + l0, n_ahead, uq0, stream) != cudaSuccess)
-      return KVSWAP_ERR_CUDA;
-    for (int l = l0; l < l0 + n_ahead; ++l) {
-      const bool probed = probe_opt != nullptr && probe_opt->layer == l;
-      const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-      int32_t* idx_l = group_idx + size_t(l) * idx_elems;
-      int32_t* nsel_l = n_selected + size_t(l) * nsel_elems;
-      if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), stream);
-      const float* uq = uq0 + size_t(l - l0) * p.B * p.Su * p.r;
-      if (score_select_from_uq(p, w, uq, layers->meta[l], idx_l, nsel_l, nullptr, ws, stream) != cudaSuccess)
-        return KVSWAP_ERR_CUDA;
-      if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), stream);
-      st = kvswap_sparse_decode(shape, ql, layers->K[l], layers->V[l], idx_l, nsel_l, out + size_t(l) * out_elems,
-                                lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes, cuda_stream);
-      if (st != KVSWAP_OK) return st;
-      if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
-    }
+  for (int l = 0; l < L; ++l) {
+    if (layers->proj[l] == nullptr || layers->meta[l] == nullptr || layers->K[l] == nullptr || layers->V[l] == nullptr)
+      return KVSWAP_ERR_NULL;
+    if (misaligned(layers->proj[l]) || misaligned(layers->meta[l])) return KVSWAP_ERR_ALIGN;
   }
-  return KVSWAP_OK;
+
+  // Schedule (Sec. 4.3, online prediction, and Sec. 4.4): a layer's groups are predicted ahead of
+  // its attention, concurrently with the layers before it.  The predictor therefore runs on a
+  // stream of its own, ahead of the attention on the caller's stream by at most `look` layers:
+  //   predictor stream:  ... wait attended[l-1-look];  score/select(l);  record selected[l]  ...
+  //   caller's stream:   ... wait selected[l];         attention(l);     record attended[l]  ...
+  // With look = 1, predictor(l) overlaps attention(l-1) only: nothing runs further ahead than a
+  // model whose layer-(l-1) input (from which the paper forms the approximate query) exists
+  // once layer l-2 is done could run.  Everything on the predictor stream is ordered after the
+  // work already in the caller's stream (fork event) and joins it again through the last
+  // selection event.
+  const int look = layers->max_lookahead > 0 ? layers->max_lookahead : kDefaultLookahead;
+  std::lock_guard<std::mutex> lock(g_step_mutex);
+  StepResources* res = nullptr;
+  if (step_resources(L, &res) != cudaSuccess) return KVSWAP_ERR_CUDA;
+  cudaStream_t pred = res->predictor;
+  if (cudaEventRecord(res->fork, stream) != cudaSuccess || cudaStreamWaitEvent(pred, res->fork, 0) != cudaSuccess)
+    return KVSWAP_ERR_CUDA;
+
+  auto enqueue_predictor = [&](int l) -> int {
+    if (l > look && cudaStreamWaitEvent(pred, res->attended[l - 1 - look], 0) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+    const bool probed = probe_opt != nullptr && probe_opt->layer == l;
+    if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), pred);
+    const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+    if (score_select_launch(p, w, ql, layers->proj[l], layers->meta[l], group_idx + size_t(l) * idx_elems,
+                            n_selected + size_t(l) * nsel_elems, nullptr, ws, pred) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+    if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), pred);
+    if (cudaEventRecord(res->selected[l], pred) != cudaSuccess) return KVSWAP_ERR_CUDA;
+    return KVSWAP_OK;
+  };
+  auto enqueue_attention = [&](int l) -> int {
+    if (cudaStreamWaitEvent(stream, res->selected[l], 0) != cudaSuccess) return KVSWAP_ERR_CUDA;
+    const bool probed = probe_opt != nullptr && probe_opt->layer == l;
+    const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+    const int r = kvswap_sparse_decode(shape, ql, layers->K[l], layers->V[l], group_idx + size_t(l) * idx_elems,
+                                       n_selected + size_t(l) * nsel_elems, out + size_t(l) * out_elems,
+                                       lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes,
+                                       cuda_stream);
+    if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
+    if (r == KVSWAP_OK && cudaEventRecord(res->attended[l], stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+    return r;
+  };
+
+  // Host order: each predictor is handed to its stream up to kHostLead layers before the
+  // attention that consumes it, never before the attention whose event it waits on.
+  const int lead = std::min(look, kHostLead);
+  int status = KVSWAP_OK;
+  int next_pred = 0;
+  for (int l = 0; l < L && status == KVSWAP_OK; ++l) {
+    while (status == KVSWAP_OK && next_pred < L && next_pred <= l + lead) status = enqueue_predictor(next_pred++);
+    if (status == KVSWAP_OK) status = enqueue_attention(l);
+  }
+  if (status != KVSWAP_OK) {
+    // a launch failed: join whatever the predictor stream was given after its last awaited event
+    if (cudaEventRecord(res->fork, pred) != cudaSuccess || cudaStreamWaitEvent(stream, res->fork, 0) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+  }
+  return status;
 }
 
 int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* layers, const void* q_host,

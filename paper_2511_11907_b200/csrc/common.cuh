@@ -29,7 +29,7 @@ struct Problem {
 
 // Partition of the caller's workspace (byte offsets, each 256-byte aligned).
 struct Workspace {
-  size_t off_uq;       // float [uq_layers, B, Su, r]  summed low-rank queries (a whole decode step computes several layers' at once)
+  size_t off_uq;       // float [B, Su, r]       summed low-rank queries
   size_t off_scores;   // float [B, S, NG]       group scores R (when the caller passes no buffer)
   size_t off_partial;  // float [B, Hq, splits, d + 2]  split-K partials (m, l, acc[d])
   size_t off_adapter;  // bf16 [H_kv, 3 r, d]       adapter split into three bf16 pieces (project_keys on tcgen05)
@@ -37,7 +37,6 @@ struct Workspace {
   int splits;          // split-K factor of sparse_decode for this shape
   int heads_per_cta;   // query heads sharing one K/V pass in sparse_decode
   int depth;           // shared-memory stages per compute warp in sparse_decode
-  int uq_layers;       // layers whose low-rank queries fit the off_uq region
 };
 
 int resolve(const kvswap_shape* s, Problem* p);            // validation; returns kvswap_status
@@ -51,10 +50,8 @@ cudaError_t launch_project_keys(const Problem& p, const void* K, const float* pr
 size_t project_keys_umma_scratch_bytes(const Problem& p);
 bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
                                   int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result);
-// Low-rank queries of up to kMaxQueryLayers layers in one launch: q [n, B, H_q, d] -> uq [n, B, Su, r].
-constexpr int kMaxQueryLayers = 64;
-cudaError_t launch_lowrank_query_layers(const Problem& p, const void* q, const float* const* proj, int n_layers,
-                                        float* uq, cudaStream_t st);
+cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* proj, float* uq,
+                                 cudaStream_t st);
 cudaError_t launch_score_pool(const Problem& p, const float* uq, const void* meta, float* scores,
                               uint32_t* err, cudaStream_t st);
 cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* group_idx,

@@ -30,16 +30,10 @@ constexpr uint32_t kFull = 0xffffffffu;
 // it (one, except for joint metadata under the all-heads scope).  256 threads = 8 slices of the
 // contraction index x 32 output columns (r <= 32), or the generic loop for larger r.
 // ------------------------------------------------------------------------------------------
-// Adapters of the layers one launch serves (blockIdx.z = layer).
-struct ProjTable { const float* proj[kMaxQueryLayers]; };
-
 template <typename Q_T>
 __global__ void __launch_bounds__(4 * kThreads)
-lowrank_query_kernel(Problem p, const Q_T* __restrict__ q_base, int64_t q_layer_stride, const ProjTable table,
-                     float* __restrict__ uq_base, int64_t uq_layer_stride) {
-  const Q_T* __restrict__ q = q_base + int64_t(blockIdx.z) * q_layer_stride;
-  const float* __restrict__ proj = table.proj[blockIdx.z];
-  float* __restrict__ uq = uq_base + int64_t(blockIdx.z) * uq_layer_stride;
+lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restrict__ proj,
+                     float* __restrict__ uq) {
   // blockDim.x = kThreads * n_grp: thread group `grp` (256 threads) takes the KV heads
   // g0 + grp, g0 + grp + n_grp, ... of the row, so that up to four heads are in flight at once.
   __shared__ float qsum[4][128];
@@ -701,28 +695,20 @@ cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, flo
 
 }  // namespace
 
-// Summed low-rank queries of `n_layers` layers in one launch: q [n, B, H_q, d], uq [n, B, Su, r].
-cudaError_t launch_lowrank_query_layers(const Problem& p, const void* q, const float* const* proj, int n_layers,
-                                        float* uq, cudaStream_t st) {
-  if (n_layers < 1 || n_layers > kMaxQueryLayers) return cudaErrorInvalidValue;
-  ProjTable table = {};
-  for (int l = 0; l < n_layers; ++l) table.proj[l] = proj[l];
-  dim3 grid(p.B, p.Su, n_layers);
+cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* proj, float* uq, cudaStream_t st) {
+  dim3 grid(p.B, p.Su);
   // One 256-thread group per KV head in flight: one group per row, up to four when a row sums
   // all KV heads (joint metadata under the all-heads scope).
   const bool joint_all = (p.Hm == 1 && p.scope == KVSWAP_SCOPE_ALL_HEADS);
   const dim3 block(kThreads * (joint_all ? std::min(4, p.Hkv) : 1));
-  const int64_t q_stride = int64_t(p.B) * p.Hq * p.d, uq_stride = int64_t(p.B) * p.Su * p.r;
   switch (p.q_dtype) {
     case KVSWAP_F32:
-      return launch_pdl(lowrank_query_kernel<float>, grid, block, 0, st, p, static_cast<const float*>(q), q_stride, table,
-                        uq, uq_stride);
+      return launch_pdl(lowrank_query_kernel<float>, grid, block, 0, st, p, static_cast<const float*>(q), proj, uq);
     case KVSWAP_BF16:
       return launch_pdl(lowrank_query_kernel<__nv_bfloat16>, grid, block, 0, st, p,
-                        static_cast<const __nv_bfloat16*>(q), q_stride, table, uq, uq_stride);
+                        static_cast<const __nv_bfloat16*>(q), proj, uq);
     default:
-      return launch_pdl(lowrank_query_kernel<__half>, grid, block, 0, st, p, static_cast<const __half*>(q), q_stride,
-                        table, uq, uq_stride);
+      return launch_pdl(lowrank_query_kernel<__half>, grid, block, 0, st, p, static_cast<const __half*>(q), proj, uq);
   }
 }
 

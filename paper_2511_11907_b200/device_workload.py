@@ -59,8 +59,8 @@ class DeviceWorkload:
     layers_resident: int                 # distinct K/V buffers (== L unless memory forced sharing)
     heavy_pos: Optional[List[torch.Tensor]] = None
 
-    def layer_tables(self) -> kv.kvswap_layers:
-        return kv.make_layers(self.K, self.V, self.meta, self.proj)
+    def layer_tables(self, max_lookahead: int = 0) -> kv.kvswap_layers:
+        return kv.make_layers(self.K, self.V, self.meta, self.proj, max_lookahead)
 
 
 def build(wl: W.Workload, meta_heads: int = 1, scope: int = W.SCOPE_KV_HEAD, device="cuda", rank_offset: int = 0,

@@ -49,6 +49,27 @@ def test_struct_layout_matches_header():
     assert ctypes.sizeof(kv.kvswap_shape) == 13 * 4 + 4 + 6 * 8   # 13 int32, padding, 6 int64
 
 
+def test_layers_struct_layout_matches_header():
+    # int32 n_layers, int32 max_lookahead, four pointers
+    assert ctypes.sizeof(kv.kvswap_layers) == 8 + 4 * ctypes.sizeof(ctypes.c_void_p)
+    assert kv.kvswap_layers.max_lookahead.offset == 4 and kv.kvswap_layers.K.offset == 8
+
+
+def test_decode_step_rejects_bad_layer_tables(lib):
+    kv._declare_step(lib)
+    s = good_shape()
+    fake = ctypes.c_void_p(4096)
+    tab = (ctypes.c_void_p * 1)(4096)
+    ptab = ctypes.cast(tab, ctypes.POINTER(ctypes.c_void_p))
+    assert lib.kvswap_decode_step(ctypes.byref(s), None, fake, fake, None, fake, fake, fake, 1 << 30, None, None) == 1
+    for bad in (kv.kvswap_layers(0, 0, ptab, ptab, ptab, ptab), kv.kvswap_layers(1, -1, ptab, ptab, ptab, ptab)):
+        assert lib.kvswap_decode_step(ctypes.byref(s), ctypes.byref(bad), fake, fake, None, fake, fake, fake,
+                                      1 << 30, None, None) == 2
+    ok = kv.kvswap_layers(1, 0, ptab, ptab, ptab, ptab)
+    assert lib.kvswap_decode_step(ctypes.byref(s), ctypes.byref(ok), fake, fake, None, fake, fake, fake, 16,
+                                  None, None) == 5        # workspace too small: refused before any launch
+
+
 def test_validation_status_codes(lib):
     assert kv.kvswap_validate_shape(good_shape()) == 0
     assert kv.kvswap_workspace_bytes(good_shape()) > 0

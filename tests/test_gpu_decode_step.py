@@ -1,6 +1,6 @@
-"""kvswap_decode_step (all layers of one decode step in one call, low-rank queries computed for
-many layers ahead of the per-layer work) gives exactly what the three per-layer calls give.
-The per-layer calls themselves are checked against the oracle in test_gpu_parity.py."""
+"""kvswap_decode_step (all layers of one decode step in one call, each layer's predictor on an
+internal stream overlapping the previous layer's attention) gives exactly what the per-layer
+calls give.  The per-layer calls themselves are checked against the oracle in test_gpu_parity.py."""
 import pytest
 import torch
 
@@ -22,7 +22,7 @@ def _step_buffers(dw):
     return out, lse, idx, nsel
 
 
-def _run_case(wl, meta_heads, scope):
+def _run_case(wl, meta_heads, scope, lookahead=0):
     dw = DW.build(wl, 1 if meta_heads == "joint" else wl.n_kv_heads, scope, walk_steps=1, reserve_bytes=1 << 30)
     assert dw.layers_resident == wl.layers
     ws = rt.alloc_workspace(dw.shape)
@@ -42,7 +42,7 @@ def _run_case(wl, meta_heads, scope):
     ws.fill_(0xFF)
     kv.kvswap_workspace_init(ws)
     out_b, lse_b, idx_b, nsel_b = _step_buffers(dw)
-    kv.kvswap_decode_step(dw.shape, dw.layer_tables(), q, out_b, lse_b, idx_b, nsel_b, ws)
+    kv.kvswap_decode_step(dw.shape, dw.layer_tables(lookahead), q, out_b, lse_b, idx_b, nsel_b, ws)
     torch.cuda.synchronize()
     assert kv.kvswap_read_device_status(ws) == 0
     assert torch.equal(nsel_a, nsel_b)
@@ -56,10 +56,29 @@ def _run_case(wl, meta_heads, scope):
     q_host = q.cpu().pin_memory()
     out_host = torch.full(out_c.shape, float("nan"), dtype=torch.float32).pin_memory()
     q_dev = torch.zeros_like(q)
-    kv.kvswap_decode_step_host(dw.shape, dw.layer_tables(), q_host, out_host, q_dev, out_c, idx_c, nsel_c, ws)
+    kv.kvswap_decode_step_host(dw.shape, dw.layer_tables(lookahead), q_host, out_host, q_dev, out_c, idx_c, nsel_c, ws)
     torch.cuda.synchronize()
     assert torch.equal(idx_a, idx_c)
     assert torch.equal(out_a.cpu(), out_host)
+
+    # repeated steps reuse the internal stream and events
+    for _ in range(3):
+        kv.kvswap_decode_step(dw.shape, dw.layer_tables(lookahead), q, out_b, lse_b, idx_b, nsel_b, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(idx_a, idx_b) and torch.equal(out_a, out_b)
+    assert kv.kvswap_read_device_status(ws) == 0
+
+
+def test_single_layer_step():
+    wl = W.CONFIGS[2].reduced("cfg2-one", n_ctx=2048 + 7, top_k=32, calib_rows=1024)
+    _run_case(wl, "joint", W.SCOPE_KV_HEAD)
+
+
+def test_decode_step_on_a_side_stream():
+    wl = W.CONFIGS[3].reduced("cfg3-side", layers=3, batch=2, n_ctx=2048, top_k=20, calib_rows=1024)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        _run_case(wl, "joint", W.SCOPE_KV_HEAD)
 
 
 @pytest.mark.parametrize("meta_heads", ["joint", "per_head"])
@@ -69,15 +88,16 @@ def test_decode_step_equals_layer_by_layer_calls(meta_heads, scope):
     _run_case(wl, meta_heads, scope)
 
 
-def test_decode_step_with_more_layers_than_one_query_launch_serves():
-    """70 layers: the low-rank queries are computed in two launches (64 layers, then 6)."""
+@pytest.mark.parametrize("lookahead", [1, 2, 5, 1000])
+def test_decode_step_over_many_layers(lookahead):
+    """70 thin layers: the two streams hand over 140 times within one step."""
     wl = W.CONFIGS[3].reduced("cfg3-deep", layers=70, batch=1, n_ctx=1024 + 3, top_k=16, calib_rows=1024,
                               n_q_heads=8, n_kv_heads=2)
-    _run_case(wl, "joint", W.SCOPE_KV_HEAD)
+    _run_case(wl, "joint", W.SCOPE_KV_HEAD, lookahead)
 
 
-def test_decode_step_when_the_workspace_holds_few_layers_of_queries():
-    """fp32, large batch x rank: one layer's low-rank queries take 256 KiB, so four layers go per launch."""
+def test_decode_step_fp32_wide_rank_per_head():
+    """fp32 everywhere, rank 128 per-head metadata, batch 64 (generic kernels on both streams)."""
     wl = W.CONFIGS[1].reduced("cfg1-wide", layers=6, batch=64, n_ctx=512, rank=128, head_dim=128, n_q_heads=32,
                               n_kv_heads=8, top_k=8, calib_rows=1536)
     _run_case(wl, "per_head", W.SCOPE_KV_HEAD)
