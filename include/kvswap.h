@@ -64,6 +64,18 @@ typedef enum { KVSWAP_F32 = 0, KVSWAP_BF16 = 1, KVSWAP_F16 = 2 } kvswap_dtype;
 typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_scope;
 
 /*
+ * kvswap_shape.flags (bit set; unknown bits are KVSWAP_ERR_SHAPE).
+ *   KVSWAP_INPUTS_SETTLED  a promise by the caller of kvswap_sparse_decode: q, group_idx and
+ *       n_selected (like K and V) are not outputs of work that may still be running when the
+ *       call's kernels start, i.e. nothing enqueued earlier in `cuda_stream` writes them, or a
+ *       full dependency (an event wait, a copy, a host synchronisation) lies in between.  The
+ *       gather kernel then starts fetching K/V rows while the previous kernel of the stream is
+ *       still finishing (programmatic dependent launch) and only waits for it before writing
+ *       its own results.  Without the flag it waits first.  Other calls ignore the flag.
+ */
+enum { KVSWAP_INPUTS_SETTLED = 1 };
+
+/*
  * Problem description shared by all calls.
  *   kv_*   strides (in elements) of K and V, both laid out [B, H_kv, N, d];
  *   meta_* strides (in elements) of the metadata, laid out [B, H_m, N, r].
@@ -76,6 +88,7 @@ typedef struct {
   int32_t batch, n_ctx, n_q_heads, n_kv_heads, head_dim; /* B, N, H_q, H_kv, d            */
   int32_t rank, meta_heads, group_size, top_k;           /* r, H_m in {1, H_kv}, G, M     */
   int32_t kv_dtype, meta_dtype, q_dtype, scope;          /* enums above                   */
+  int32_t flags;                                         /* 0 or KVSWAP_INPUTS_SETTLED    */
   int64_t kv_stride_b, kv_stride_h, kv_stride_n;
   int64_t meta_stride_b, meta_stride_h, meta_stride_n;
 } kvswap_shape;
@@ -187,8 +200,8 @@ int kvswap_sparse_decode_static(const kvswap_shape* shape, const void* q, const 
  * HOST array of L DEVICE pointers: K[l], V[l] are [B, H_kv, N, d]; meta[l] is [B, H_m, N, r];
  * proj[l] is [H_kv, d, r] fp32.  max_lookahead bounds how many layers kvswap_decode_step's
  * predictor may run ahead of its attention: 1 = layer l is predicted while layer l-1 is attended
- * (what a model allows, whose layer-l prediction needs the input of layer l-1); 0 = the
- * library's default (3).  Negative values are KVSWAP_ERR_SHAPE.
+ * (what a model allows, whose layer-l prediction needs the input of layer l-1); 0 = no limit.
+ * Negative values are KVSWAP_ERR_SHAPE.
  */
 typedef struct {
   int32_t n_layers;

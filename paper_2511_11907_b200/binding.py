@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_PKG, "libkvswap.so")
 
 KVSWAP_F32, KVSWAP_BF16, KVSWAP_F16 = 0, 1, 2
 KVSWAP_SCOPE_KV_HEAD, KVSWAP_SCOPE_ALL_HEADS = 0, 1
+KVSWAP_INPUTS_SETTLED = 1      # kvswap_shape.flags
 
 
 class KVSwapError(RuntimeError):
@@ -27,8 +28,14 @@ class KVSwapError(RuntimeError):
 class kvswap_shape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "batch", "n_ctx", "n_q_heads", "n_kv_heads", "head_dim", "rank", "meta_heads", "group_size",
-        "top_k", "kv_dtype", "meta_dtype", "q_dtype", "scope")] + [(n, ctypes.c_int64) for n in (
+        "top_k", "kv_dtype", "meta_dtype", "q_dtype", "scope", "flags")] + [(n, ctypes.c_int64) for n in (
         "kv_stride_b", "kv_stride_h", "kv_stride_n", "meta_stride_b", "meta_stride_h", "meta_stride_n")]
+
+    def with_flags(self, flags: int) -> "kvswap_shape":
+        """A copy of the shape with `flags` set."""
+        other = kvswap_shape.from_buffer_copy(self)
+        other.flags = int(flags)
+        return other
 
     @property
     def n_scopes(self) -> int:
@@ -81,9 +88,9 @@ def status_string(status: int) -> str:
 
 def make_shape(*, batch, n_ctx, n_q_heads, n_kv_heads, head_dim, rank, meta_heads, group_size, top_k,
                kv_dtype, meta_dtype, q_dtype, scope=KVSWAP_SCOPE_KV_HEAD, kv_strides=(0, 0, 0),
-               meta_strides=(0, 0, 0)) -> kvswap_shape:
+               meta_strides=(0, 0, 0), flags=0) -> kvswap_shape:
     return kvswap_shape(batch, n_ctx, n_q_heads, n_kv_heads, head_dim, rank, meta_heads, group_size, top_k,
-                        kv_dtype, meta_dtype, q_dtype, scope, *kv_strides, *meta_strides)
+                        kv_dtype, meta_dtype, q_dtype, scope, flags, *kv_strides, *meta_strides)
 
 
 def _ptr(t) -> Optional[int]:
@@ -162,7 +169,7 @@ class kvswap_probe(ctypes.Structure):
 def make_layers(K, V, meta, proj, max_lookahead: int = 0) -> kvswap_layers:
     """Pointer tables for lists of per-layer device tensors.  The returned struct keeps the
     tensors and the tables alive.  max_lookahead: layers the predictor of kvswap_decode_step may
-    run ahead of the attention (0 = library default, 1 = one layer, as a model allows)."""
+    run ahead of the attention (0 = no limit, 1 = one layer, as a model allows)."""
     n = len(K)
     assert len(V) == n and len(meta) == n and len(proj) == n
 

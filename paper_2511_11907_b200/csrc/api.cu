@@ -27,6 +27,7 @@ int resolve(const kvswap_shape* s, Problem* p) {
   if (s->n_q_heads % s->n_kv_heads != 0) return KVSWAP_ERR_SHAPE;
   if (s->meta_heads != 1 && s->meta_heads != s->n_kv_heads) return KVSWAP_ERR_SHAPE;
   if (s->scope != KVSWAP_SCOPE_KV_HEAD && s->scope != KVSWAP_SCOPE_ALL_HEADS) return KVSWAP_ERR_SHAPE;
+  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED)) != 0) return KVSWAP_ERR_SHAPE;
   if (s->n_ctx > (1 << 30) || s->batch > 65535 || s->n_q_heads > 4096) return KVSWAP_ERR_SHAPE;
   const int ekv = dtype_bytes(s->kv_dtype), em = dtype_bytes(s->meta_dtype), eq = dtype_bytes(s->q_dtype);
   if (ekv == 0 || em == 0 || eq == 0) return KVSWAP_ERR_DTYPE;
@@ -41,6 +42,7 @@ int resolve(const kvswap_shape* s, Problem* p) {
   p->B = s->batch; p->N = s->n_ctx; p->Hq = s->n_q_heads; p->Hkv = s->n_kv_heads; p->d = s->head_dim;
   p->r = s->rank; p->Hm = s->meta_heads; p->G = s->group_size; p->M = s->top_k;
   p->kv_dtype = s->kv_dtype; p->meta_dtype = s->meta_dtype; p->q_dtype = s->q_dtype; p->scope = s->scope;
+  p->flags = s->flags;
 
   p->kv_sn = s->kv_stride_n ? s->kv_stride_n : p->d;
   p->kv_sh = s->kv_stride_h ? s->kv_stride_h : int64_t(p->N) * p->kv_sn;
@@ -203,7 +205,6 @@ struct StepResources {
   std::vector<cudaEvent_t> attended;     // attended[l]: layer l's attention output is written
 };
 constexpr int kMaxDevices = 64;
-constexpr int kDefaultLookahead = 3;   // layers the predictor may run ahead when the caller sets no limit
 constexpr int kHostLead = 3;           // layers by which the host enqueues the predictor ahead of the attention
 std::mutex g_step_mutex;
 StepResources g_step[kMaxDevices];
@@ -266,15 +267,24 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
 
   // Schedule (Sec. 4.3, online prediction, and Sec. 4.4): a layer's groups are predicted ahead of
   // its attention, concurrently with the layers before it.  The predictor therefore runs on a
-  // stream of its own, ahead of the attention on the caller's stream by at most `look` layers:
+  // stream of its own, ahead of the attention on the caller's stream by at most `look` layers
+  // (any number when the caller sets no limit):
   //   predictor stream:  ... wait attended[l-1-look];  score/select(l);  record selected[l]  ...
   //   caller's stream:   ... wait selected[l];         attention(l);     record attended[l]  ...
   // With look = 1, predictor(l) overlaps attention(l-1) only: nothing runs further ahead than a
   // model whose layer-(l-1) input (from which the paper forms the approximate query) exists
-  // once layer l-2 is done could run.  Everything on the predictor stream is ordered after the
-  // work already in the caller's stream (fork event) and joins it again through the last
-  // selection event.
-  const int look = layers->max_lookahead > 0 ? layers->max_lookahead : kDefaultLookahead;
+  // once layer l-2 is done could run.  With look >= 2 the caller's stream waits for two layers'
+  // selections at a time, so that every second attention follows the previous one without a
+  // stream-level wait in between and, its inputs being settled, starts fetching while that one
+  // is still finishing.  Everything on the predictor stream is ordered after the work already
+  // in the caller's stream (fork event) and joins it again through the last selection event.
+  const bool bounded = layers->max_lookahead > 0 && layers->max_lookahead < L;
+  const int look = bounded ? layers->max_lookahead : L;
+  const int join = look >= 2 ? 2 : 1;          // layers of attention per wait on the predictor
+  // q is an input of the step and each selection is awaited through its event before the
+  // attention that reads it is launched: the attention's inputs are settled.
+  kvswap_shape shape_settled = *shape;
+  shape_settled.flags |= KVSWAP_INPUTS_SETTLED;
   std::lock_guard<std::mutex> lock(g_step_mutex);
   StepResources* res = nullptr;
   if (step_resources(L, &res) != cudaSuccess) return KVSWAP_ERR_CUDA;
@@ -283,7 +293,7 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
     return KVSWAP_ERR_CUDA;
 
   auto enqueue_predictor = [&](int l) -> int {
-    if (l > look && cudaStreamWaitEvent(pred, res->attended[l - 1 - look], 0) != cudaSuccess)
+    if (bounded && l > look && cudaStreamWaitEvent(pred, res->attended[l - 1 - look], 0) != cudaSuccess)
       return KVSWAP_ERR_CUDA;
     const bool probed = probe_opt != nullptr && probe_opt->layer == l;
     if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), pred);
@@ -296,25 +306,30 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
     return KVSWAP_OK;
   };
   auto enqueue_attention = [&](int l) -> int {
-    if (cudaStreamWaitEvent(stream, res->selected[l], 0) != cudaSuccess) return KVSWAP_ERR_CUDA;
+    if (l % join == 0 &&
+        cudaStreamWaitEvent(stream, res->selected[std::min(L - 1, l + join - 1)], 0) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
     const bool probed = probe_opt != nullptr && probe_opt->layer == l;
     const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-    const int r = kvswap_sparse_decode(shape, ql, layers->K[l], layers->V[l], group_idx + size_t(l) * idx_elems,
+    const int r = kvswap_sparse_decode(&shape_settled, ql, layers->K[l], layers->V[l], group_idx + size_t(l) * idx_elems,
                                        n_selected + size_t(l) * nsel_elems, out + size_t(l) * out_elems,
                                        lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes,
                                        cuda_stream);
     if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
-    if (r == KVSWAP_OK && cudaEventRecord(res->attended[l], stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+    if (bounded && r == KVSWAP_OK && cudaEventRecord(res->attended[l], stream) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
     return r;
   };
 
-  // Host order: each predictor is handed to its stream up to kHostLead layers before the
-  // attention that consumes it, never before the attention whose event it waits on.
-  const int lead = std::min(look, kHostLead);
+  // Host order: a predictor is handed to its stream before the wait on its selection is enqueued
+  // (join - 1 layers ahead at least), up to kHostLead layers ahead of the attention that consumes
+  // it, and never before the attention whose event it waits on (look - join + 1 at most).
+  const int lead = std::max(join - 1, std::min(look - join + 1, kHostLead));
   int status = KVSWAP_OK;
   int next_pred = 0;
   for (int l = 0; l < L && status == KVSWAP_OK; ++l) {
-    while (status == KVSWAP_OK && next_pred < L && next_pred <= l + lead) status = enqueue_predictor(next_pred++);
+    while (status == KVSWAP_OK && next_pred < L && next_pred <= l - l % join + lead)
+      status = enqueue_predictor(next_pred++);
     if (status == KVSWAP_OK) status = enqueue_attention(l);
   }
   if (status != KVSWAP_OK) {

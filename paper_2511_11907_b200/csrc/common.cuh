@@ -18,6 +18,7 @@ constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs; grids are sized in multi
 struct Problem {
   int B, N, Hq, Hkv, d, r, Hm, G, M;
   int kv_dtype, meta_dtype, q_dtype, scope;
+  int flags;   // KVSWAP_INPUTS_SETTLED
   int64_t kv_sb, kv_sh, kv_sn;
   int64_t meta_sb, meta_sh, meta_sn;
   int rho;   // H_q / H_kv

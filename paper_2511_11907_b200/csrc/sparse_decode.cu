@@ -430,8 +430,11 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   const int h0 = g * p.rho + hc * RH;                          // first query head of this CTA
   const int srow = (p.scope == KVSWAP_SCOPE_KV_HEAD) ? g : 0;
 
-  // Everything below may depend on the previous kernel in the stream.
-  pdl_wait();
+  // Everything below may depend on the previous kernel in the stream -- unless the caller has
+  // promised that q and the selection are settled: then only this kernel's writes (the partials,
+  // which the previous launch's combine may still be reading) have to wait for it.
+  const bool settled = (p.flags & KVSWAP_INPUTS_SETTLED) != 0;
+  if (!settled) pdl_wait();
   pdl_trigger();
 
   // The virtual token list is laid out for M selected groups, whatever n_selected says (slots of
@@ -538,6 +541,7 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   float* sm_acc = sm_l + kWarps * 8;                                // [kWarps][RH][D]
   eng.store(sm_m + warp * 8, sm_l + warp * 8, sm_acc + warp * RH * D);
   __syncthreads();
+  if (settled) pdl_wait();
   for (int i = threadIdx.x; i < RH * D; i += kThreads) {
     const int hh = i / D, c = i % D;
     float mx = -INFINITY;
@@ -568,8 +572,10 @@ __global__ void __launch_bounds__(D)
 combine_kernel(const float* __restrict__ partial, float* __restrict__ out, float* __restrict__ lse, int splits) {
   __shared__ float w_s[kMaxSplits];
   __shared__ float norm_s[2];                  // 1 / sum of weights (or 0), lse
-  pdl_wait();
+  // The next kernel of the stream may start its own prologue at once; this one needs the
+  // partials of the gather kernel before it.
   pdl_trigger();
+  pdl_wait();
   const int64_t bh = blockIdx.x;
   const float* src = partial + bh * splits * (D + 2);
   const int c = threadIdx.x;

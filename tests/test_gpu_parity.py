@@ -270,6 +270,30 @@ def test_sparse_decode_accepts_any_valid_index_list():
     assert np.abs(out - out_o).max() <= 1e-5
 
 
+@pytest.mark.parametrize("which", ["cfg1", "cfg3-small", "cfg4-small", "cfg5-small"])
+def test_sparse_decode_with_settled_inputs_matches_the_default_mode(which):
+    """KVSWAP_INPUTS_SETTLED only moves the wait for the previous kernel: launched back to back
+    without host synchronisation (so that consecutive launches overlap), every launch still
+    returns exactly what the default mode returns."""
+    wl = W.CONFIGS[1] if which == "cfg1" else W.REDUCED[int(which[3])]
+    li = W.make_layer(wl, 0, 1)
+    dl = DeviceLayer(li, KV)
+    dl.project()
+    dl.score_select()
+    out_ref, lse_ref = dl.sparse_decode()
+    settled = dl.shape.with_flags(kv.KVSWAP_INPUTS_SETTLED)
+    outs = [torch.full_like(dl.out, float("nan")) for _ in range(6)]
+    lses = [torch.full_like(dl.lse, float("nan")) for _ in range(6)]
+    torch.cuda.synchronize()
+    for o, l_ in zip(outs, lses):
+        kv.kvswap_sparse_decode(settled, dl.q, dl.K, dl.V, dl.idx, dl.nsel, o, l_, dl.ws)
+    torch.cuda.synchronize()
+    assert kv.kvswap_read_device_status(dl.ws) == 0
+    for o, l_ in zip(outs, lses):
+        assert np.array_equal(o.cpu().numpy(), out_ref)
+        assert np.array_equal(l_.cpu().numpy(), lse_ref)
+
+
 def test_no_token_attended_gives_zero_output_and_minus_inf_lse():
     wl = small(n_ctx=40)
     li = W.make_layer(wl, 0, 1)
