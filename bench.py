@@ -318,14 +318,16 @@ def run_ours(args, wl):
         return a.elapsed_time(b) / (reps * L), reps * L
 
     q0 = dw.q_walk[0]
-    sel_call_ms, sel_calls = per_call_ms(lambda l: kv.kvswap_score_select(
-        shape, q0[l], dw.proj[l], dw.meta[l], idx[l], nsel[l], None, ws))
     # the selections are in place before these calls are enqueued: the launch configuration of the step
     # (KVSWAP_INPUTS_SETTLED, consecutive launches overlap their prologue and tail); the default mode,
     # which waits for the previous kernel first, is timed beside it
     shape_settled = shape.with_flags(kv.KVSWAP_INPUTS_SETTLED)
     dec_call_ms, dec_calls = per_call_ms(lambda l: kv.kvswap_sparse_decode(
         shape_settled, q0[l], dw.K[l], dw.V[l], idx[l], nsel[l], out[l], None, ws))
+    sel_call_ms, sel_calls = per_call_ms(lambda l: kv.kvswap_score_select(
+        shape_settled, q0[l], dw.proj[l], dw.meta[l], idx[l], nsel[l], None, ws))
+    sel_wait_ms, _ = per_call_ms(lambda l: kv.kvswap_score_select(
+        shape, q0[l], dw.proj[l], dw.meta[l], idx[l], nsel[l], None, ws))
     dec_wait_ms, _ = per_call_ms(lambda l: kv.kvswap_sparse_decode(
         shape, q0[l], dw.K[l], dw.V[l], idx[l], nsel[l], out[l], None, ws))
 
@@ -413,7 +415,10 @@ def run_ours(args, wl):
         "roofline_score_select": {"bound": "hbm", "kernel": "kvswap_score_select (lowrank_query + score_pool + topk)",
                                   "achieved": sel_gbs, "peak": peak, "unit": "GB/s", "frac": sel_gbs / peak,
                                   "algorithmic_bytes_per_launch": select_bytes, "avg_ms": sel_ms,
-                                  "launches_timed": sel_calls, "in_step_probe_ms": statistics.mean(select_ms)},
+                                  "launches_timed": sel_calls,
+                                  "avg_ms_waiting_for_previous_kernel": sel_wait_ms,
+                                  "frac_waiting_for_previous_kernel": select_bytes / sel_wait_ms / 1e6 / peak,
+                                  "in_step_probe_ms": statistics.mean(select_ms)},
         "prefill": {"project_keys_ms_all_layers": prefill_ms,
                     "keys_projected_per_sec": keys_per_step / prefill_ms * 1e3,
                     "read_gbs": L * wl.batch * wl.n_kv_heads * wl.n_ctx * wl.head_dim * esz[wl.kv_dtype] / prefill_ms / 1e6},

@@ -65,13 +65,14 @@ typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_sco
 
 /*
  * kvswap_shape.flags (bit set; unknown bits are KVSWAP_ERR_SHAPE).
- *   KVSWAP_INPUTS_SETTLED  a promise by the caller of kvswap_sparse_decode: q, group_idx and
- *       n_selected (like K and V) are not outputs of work that may still be running when the
- *       call's kernels start, i.e. nothing enqueued earlier in `cuda_stream` writes them, or a
- *       full dependency (an event wait, a copy, a host synchronisation) lies in between.  The
- *       gather kernel then starts fetching K/V rows while the previous kernel of the stream is
- *       still finishing (programmatic dependent launch) and only waits for it before writing
- *       its own results.  Without the flag it waits first.  Other calls ignore the flag.
+ *   KVSWAP_INPUTS_SETTLED  a promise by the caller of kvswap_score_select or
+ *       kvswap_sparse_decode: the call's inputs (q; for kvswap_sparse_decode also group_idx and
+ *       n_selected; K, V, proj and the metadata always) are not outputs of work that may still
+ *       be running when the call's kernels start, i.e. nothing enqueued earlier in `cuda_stream`
+ *       writes them, or a full dependency (an event wait, a copy, a host synchronisation) lies
+ *       in between.  The first kernel of the call then starts while the previous kernel of the
+ *       stream is still finishing (programmatic dependent launch) and only waits for it before
+ *       writing its own results.  Without the flag it waits first.  Results are the same.
  */
 enum { KVSWAP_INPUTS_SETTLED = 1 };
 

@@ -281,10 +281,13 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
   const bool bounded = layers->max_lookahead > 0 && layers->max_lookahead < L;
   const int look = bounded ? layers->max_lookahead : L;
   const int join = look >= 2 ? 2 : 1;          // layers of attention per wait on the predictor
-  // q is an input of the step and each selection is awaited through its event before the
-  // attention that reads it is launched: the attention's inputs are settled.
+  // q is an input of the step (the fork event orders both streams after whatever produced it) and
+  // each selection is awaited through its event before the attention that reads it is launched:
+  // the inputs of both the predictor and the attention are settled.
   kvswap_shape shape_settled = *shape;
   shape_settled.flags |= KVSWAP_INPUTS_SETTLED;
+  Problem p_settled = p;
+  p_settled.flags |= KVSWAP_INPUTS_SETTLED;
   std::lock_guard<std::mutex> lock(g_step_mutex);
   StepResources* res = nullptr;
   if (step_resources(L, &res) != cudaSuccess) return KVSWAP_ERR_CUDA;
@@ -298,7 +301,7 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
     const bool probed = probe_opt != nullptr && probe_opt->layer == l;
     if (probed && probe_opt->ev_begin) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_begin), pred);
     const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-    if (score_select_launch(p, w, ql, layers->proj[l], layers->meta[l], group_idx + size_t(l) * idx_elems,
+    if (score_select_launch(p_settled, w, ql, layers->proj[l], layers->meta[l], group_idx + size_t(l) * idx_elems,
                             n_selected + size_t(l) * nsel_elems, nullptr, ws, pred) != cudaSuccess)
       return KVSWAP_ERR_CUDA;
     if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), pred);

@@ -38,7 +38,10 @@ lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restri
   // g0 + grp, g0 + grp + n_grp, ... of the row, so that up to four heads are in flight at once.
   __shared__ float qsum[4][128];
   __shared__ float red[4 * kThreads];
-  pdl_wait();
+  // With the query settled (KVSWAP_INPUTS_SETTLED) only the write of the result has to wait for
+  // the previous kernel of the stream, whose predecessors may still be reading the buffer.
+  const bool settled = (p.flags & KVSWAP_INPUTS_SETTLED) != 0;
+  if (!settled) pdl_wait();
   pdl_trigger();
   const int b = blockIdx.x, row = blockIdx.y;
   const int tid = threadIdx.x % kThreads, grp = threadIdx.x / kThreads, n_grp = blockDim.x / kThreads;
@@ -94,6 +97,7 @@ lowrank_query_kernel(Problem p, const Q_T* __restrict__ q, const float* __restri
   }
   red[threadIdx.x] = (part < parts) ? acc : 0.f;
   __syncthreads();
+  if (settled) pdl_wait();
   if (threadIdx.x < p.r) {
     float s = 0.f;
     for (int gq = 0; gq < n_grp; ++gq)

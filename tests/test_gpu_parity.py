@@ -294,6 +294,32 @@ def test_sparse_decode_with_settled_inputs_matches_the_default_mode(which):
         assert np.array_equal(l_.cpu().numpy(), lse_ref)
 
 
+@pytest.mark.parametrize("which", ["cfg1", "cfg3-small", "cfg4-small", "cfg5-small"])
+@pytest.mark.parametrize("meta_heads", ["joint", "per_head"])
+def test_score_select_with_settled_inputs_matches_the_default_mode(which, meta_heads):
+    """Back-to-back launches (no host synchronisation in between) with KVSWAP_INPUTS_SETTLED give
+    the selections and scores of the default mode."""
+    wl = W.CONFIGS[1] if which == "cfg1" else W.REDUCED[int(which[3])]
+    li = W.make_layer(wl, 0, 1 if meta_heads == "joint" else wl.n_kv_heads)
+    dl = DeviceLayer(li, KV)
+    dl.project()
+    idx_ref, nsel_ref, scores_ref = dl.score_select()
+    settled = dl.shape.with_flags(kv.KVSWAP_INPUTS_SETTLED)
+    idxs = [torch.full_like(dl.idx, -7) for _ in range(6)]
+    nsels = [torch.full_like(dl.nsel, -7) for _ in range(6)]
+    scores = [torch.full_like(dl.scores, float("nan")) for _ in range(6)]
+    torch.cuda.synchronize()
+    for i in range(6):
+        kv.kvswap_score_select(settled, dl.q, dl.proj, dl.meta, idxs[i], nsels[i], scores[i] if i % 2 else None, dl.ws)
+    torch.cuda.synchronize()
+    assert kv.kvswap_read_device_status(dl.ws) == 0
+    for i in range(6):
+        assert np.array_equal(idxs[i].cpu().numpy(), idx_ref)
+        assert np.array_equal(nsels[i].cpu().numpy(), nsel_ref)
+        if i % 2:
+            assert np.array_equal(scores[i].cpu().numpy(), scores_ref)
+
+
 def test_no_token_attended_gives_zero_output_and_minus_inf_lse():
     wl = small(n_ctx=40)
     li = W.make_layer(wl, 0, 1)
