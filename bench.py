@@ -37,7 +37,7 @@ UNIT = "steps/s"
 # kernel, from the ncu capture summarised in profiles/decode_kernels_config5_one_layer.md (taken at
 # full config-5 shapes on one layer; the traffic of a launch does not depend on the layer count).
 # None for workloads that were not captured.  Key: (config, metadata layout, scope).
-NCU_TRAFFIC = {(5, "joint", "kv_head"): 134444800 + 4012032}
+NCU_TRAFFIC = {(5, "joint", "kv_head"): 134455808 + 3698688}
 
 
 def parse_args():
