@@ -174,3 +174,26 @@ def attend(q, K, V, idx, G, scope="kv_head", return_probs=False):
     if return_probs:
         return out, lse, probs
     return out, lse
+
+
+# ------------------------------------------------------------------------------------------
+# O7  New KV entries: rolling buffer, flush of a completed group                 (Sec. 4.4.1)
+# ------------------------------------------------------------------------------------------
+def append_kv(K, V, meta, k_new, v_new, proj, G, meta_dtype="f16"):
+    """One generated token joins the cache.  Its entries k_new, v_new [B, H_kv, d] are appended to
+    the rolling buffer, i.e. become token N of K and V (the attention always covers the
+    incomplete last group, see `attend`).  The predictor cannot rank them until their group is
+    complete: only when the N+1 tokens end a group of G are the group's G rows compressed
+    (O1) and appended to the compact cache.  `meta` holds rows of complete groups only,
+    [B, H_m, floor(N/G) G, r]; H_m is taken from it.  Returns (K', V', meta', flushed)."""
+    B, Hkv, N, d = K.shape
+    if meta.shape[2] != (N // G) * G:
+        raise ValueError("meta must hold exactly the rows of the complete groups")
+    K2 = np.concatenate([K, k_new[:, :, None, :].astype(K.dtype)], axis=2)
+    V2 = np.concatenate([V, v_new[:, :, None, :].astype(V.dtype)], axis=2)
+    flushed = (N + 1) % G == 0
+    if flushed:
+        rows = project_keys(K2[:, :, N + 1 - G:N + 1], proj, meta.shape[1], meta_dtype)
+        meta = np.concatenate([meta, rows.astype(meta.dtype)], axis=2)
+    return K2, V2, meta, flushed
+

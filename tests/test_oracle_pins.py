@@ -438,3 +438,119 @@ def test_pins_detect_planted_mistakes(monkeypatch):
     monkeypatch.setattr(O, "attend", no_tail)
     assert fails(test_sparse_attention_equals_dense_attention_over_the_selected_tokens)
     monkeypatch.setattr(O, "attend", real_attend)
+
+
+# ------------------------------------------------------------------------------------------
+# O7  rolling-buffer append and group flush (Sec. 4.4.1)
+# ------------------------------------------------------------------------------------------
+def _grow(K0, V0, k_rows, v_rows, proj, G, meta_heads, meta_dtype="f64"):
+    """Start from a context of K0.shape[2] tokens and append k_rows[t], v_rows[t] one by one."""
+    N0 = K0.shape[2]
+    meta = O.project_keys(K0[:, :, :N0 // G * G], proj, meta_heads, meta_dtype)
+    K, V, flushes = K0, V0, []
+    for t in range(len(k_rows)):
+        K, V, meta, fl = O.append_kv(K, V, meta, k_rows[t], v_rows[t], proj, G, meta_dtype)
+        flushes.append(fl)
+    return K, V, meta, flushes
+
+
+def test_append_hand_worked_example():
+    """G = 2, one head, d = r = 2, identity adapter: the compact cache is the K rows of the complete
+    groups, written out by hand."""
+    K0 = np.array([[[[1., 2.], [3., 4.], [5., 6.]]]])              # N = 3: one group + one buffered token
+    V0 = -K0
+    proj = np.eye(2)[None]
+    new_k = [np.array([[[7., 8.]]]), np.array([[[9., 10.]]]), np.array([[[11., 12.]]])]
+    new_v = [-k for k in new_k]
+    K, V, meta, flushes = _grow(K0, V0, new_k, new_v, proj, 2, 1)
+    assert flushes == [True, False, True]                           # N+1 = 4, 5, 6
+    assert np.array_equal(K[0, 0], [[1, 2], [3, 4], [5, 6], [7, 8], [9, 10], [11, 12]])
+    assert np.array_equal(V, -K)
+    assert np.array_equal(meta[0, 0], [[1, 2], [3, 4], [5, 6], [7, 8], [9, 10], [11, 12]])
+    K, V, meta, fl = O.append_kv(K, V, meta, np.array([[[13., 14.]]]), np.array([[[0., 0.]]]), proj, 2, "f64")
+    assert not fl and meta.shape[2] == 6 and K.shape[2] == 7        # token 6 waits in the rolling buffer
+
+
+@pytest.mark.parametrize("meta_heads", [1, 3])
+@pytest.mark.parametrize("G,N0,steps", [(4, 9, 11), (3, 6, 7), (1, 2, 3), (5, 1, 9)])
+def test_incremental_compact_cache_equals_compressing_the_grown_context(meta_heads, G, N0, steps):
+    """Row independence of O1: growing token by token gives the compact cache of the grown
+    context, cut at its last complete group; flushes happen exactly when a group completes."""
+    rng = np.random.default_rng(5)
+    B, Hkv, d, r = 2, 3, 4, 2
+    K0, V0 = _dyadic(rng, (B, Hkv, N0, d)), _dyadic(rng, (B, Hkv, N0, d))
+    proj = _dyadic(rng, (Hkv, d, r))
+    k_rows, v_rows = _dyadic(rng, (steps, B, Hkv, d)), _dyadic(rng, (steps, B, Hkv, d))
+    K, V, meta, flushes = _grow(K0, V0, k_rows, v_rows, proj, G, meta_heads)
+    N = N0 + steps
+    assert K.shape[2] == N and np.array_equal(K[:, :, N0:], np.moveaxis(k_rows, 0, 2))
+    assert np.array_equal(V[:, :, N0:], np.moveaxis(v_rows, 0, 2))
+    assert flushes == [(N0 + t + 1) % G == 0 for t in range(steps)]
+    want = O.project_keys(K[:, :, :N // G * G], proj, meta_heads, "f64")
+    assert meta.shape == want.shape and np.array_equal(meta, want)
+
+
+def test_appended_token_is_attended_at_once_and_ranked_only_after_its_group_completes():
+    """The rolling buffer lets a new entry take part in attention immediately (a key aligned with
+    the query and far larger than all others takes all the weight), while the predictor sees it
+    only once its group has been flushed."""
+    rng = np.random.default_rng(11)
+    B, Hq, Hkv, d, r, G, N0 = 1, 2, 1, 4, 4, 4, 8                   # two complete groups
+    K0, V0 = _dyadic(rng, (B, Hkv, N0, d)), _dyadic(rng, (B, Hkv, N0, d))
+    proj = np.eye(d)[None]
+    q = np.zeros((B, Hq, d)); q[:, :, 0] = 1.0
+    hot_k = np.zeros((B, Hkv, d)); hot_k[:, :, 0] = 400.0
+    hot_v = np.full((B, Hkv, d), 7.0)
+    meta = O.project_keys(K0, proj, 1, "f64")
+    K, V, meta, fl = O.append_kv(K0, V0, meta, hot_k, hot_v, proj, G, "f64")
+    assert not fl
+    out, _ = O.attend(q, K, V, np.zeros((B, 1, 0), dtype=np.int32), G)        # nothing selected: tail only
+    assert np.allclose(out, 7.0, atol=1e-12)
+    idx, R = O.score_select(q, proj, meta, G, 1)
+    assert R.shape[2] == 2                                           # the new token is in no group yet
+    for t in range(3):                                               # three cold tokens complete group 2
+        K, V, meta, fl = O.append_kv(K, V, meta, np.zeros((B, Hkv, d)), np.zeros((B, Hkv, d)), proj, G, "f64")
+    assert fl
+    idx, R = O.score_select(q, proj, meta, G, 1)
+    assert R.shape[2] == 3 and idx[0, 0, 0] == 2 and R[0, 0, 2] == pytest.approx(2 * 400.0)
+
+
+def test_planted_mistakes_in_append_are_caught(monkeypatch):
+    real = O.append_kv
+
+    def fails(test, *args):
+        try:
+            test(*args)
+        except AssertionError:
+            return True
+        except ValueError:
+            return True
+        return False
+
+    def flush_one_late(K, V, meta, k_new, v_new, proj, G, meta_dtype="f16"):   # tests N % G, not (N+1) % G
+        K2, V2, m2, fl = real(K, V, meta, k_new, v_new, proj, G, meta_dtype)
+        if fl:
+            return K2, V2, meta, False
+        if K.shape[2] % G == 0 and K.shape[2] // G * G > meta.shape[2]:
+            rows = O.project_keys(K[:, :, K.shape[2] - G:], proj, meta.shape[1], meta_dtype)
+            return K2, V2, np.concatenate([meta, rows], axis=2), True
+        return K2, V2, meta, False
+    monkeypatch.setattr(O, "append_kv", flush_one_late)
+    assert fails(test_append_hand_worked_example)
+
+    def wrong_rows(K, V, meta, k_new, v_new, proj, G, meta_dtype="f16"):       # compresses the G rows before the new one
+        K2, V2, m2, fl = real(K, V, meta, k_new, v_new, proj, G, meta_dtype)
+        if fl:
+            N = K.shape[2]
+            rows = O.project_keys(K2[:, :, N - G:N], proj, meta.shape[1], meta_dtype)
+            m2 = np.concatenate([meta, rows], axis=2)
+        return K2, V2, m2, fl
+    monkeypatch.setattr(O, "append_kv", wrong_rows)
+    assert fails(test_incremental_compact_cache_equals_compressing_the_grown_context, 1, 4, 9, 11)
+
+    def v_gets_k(K, V, meta, k_new, v_new, proj, G, meta_dtype="f16"):
+        return real(K, V, meta, k_new, k_new, proj, G, meta_dtype)
+    monkeypatch.setattr(O, "append_kv", v_gets_k)
+    assert fails(test_appended_token_is_attended_at_once_and_ranked_only_after_its_group_completes)
+    monkeypatch.setattr(O, "append_kv", real)
+
