@@ -131,6 +131,23 @@ int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* p
                         void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * New KV entries (Sec. 4.4.1, rolling buffer).  shape->n_ctx is the context length N BEFORE the
+ * call.  k_new, v_new [B, H_kv, d] kv_dtype (dense, device) are written to token row N of K and
+ * V; the rows past the last complete group are the rolling buffer, which kvswap_sparse_decode
+ * always attends, so the new token takes part in the next attention at once.  When the N + 1
+ * tokens end a group ((N + 1) % G == 0) the group is "flushed": its G rows of the compact cache,
+ * meta[.., N+1-G .. N, ..] = K_lr of those tokens (Sec. 4.2), are built, and from then on
+ * kvswap_score_select (called with n_ctx = N + 1) ranks the group.  *flushed_opt (host, may be
+ * NULL) is set to 1 when that happened, else 0; it depends on N and G only.
+ * The store needs room for the row: kv_stride_h and meta_stride_h must be given (not 0) and
+ * cover at least N + 1 rows, else KVSWAP_ERR_SHAPE; nothing is reallocated or moved.  After
+ * the call the caller describes the context with n_ctx = N + 1 and the same strides.
+ * Asynchronous on `cuda_stream`; needs no workspace.
+ */
+int kvswap_append_kv(const kvswap_shape* shape, const void* k_new, const void* v_new, void* K, void* V,
+                     const float* proj, void* meta, int32_t* flushed_opt, void* cuda_stream);
+
+/*
  * Grouped critical-KV prediction (Eq. 1 and "Scoring and selection", Sec. 4.3).
  * For every sequence b and selection scope s:
  *   T[b,s,n] = sum_{h in scope s} (q[b,h,:] . proj[g(h)]) . meta[b, m(g(h)), n, :]   (raw logits:

@@ -66,6 +66,8 @@ def load() -> ctypes.CDLL:
     lib.kvswap_validate_shape.argtypes = [P]
     lib.kvswap_project_keys.restype = ctypes.c_int
     lib.kvswap_project_keys.argtypes = [P, V, V, V, I32, I32, V, SZ, V]
+    lib.kvswap_append_kv.restype = ctypes.c_int
+    lib.kvswap_append_kv.argtypes = [P, V, V, V, V, V, V, ctypes.POINTER(ctypes.c_int32), V]
     lib.kvswap_score_select.restype = ctypes.c_int
     lib.kvswap_score_select.argtypes = [P, V, V, V, V, V, V, V, SZ, V]
     lib.kvswap_sparse_decode.restype = ctypes.c_int
@@ -121,6 +123,14 @@ def kvswap_project_keys(shape, K, proj, meta_out, n_begin, n_end, ws, stream=Non
     _check(load().kvswap_project_keys(ctypes.byref(shape), _ptr(K), _ptr(proj), _ptr(meta_out), int(n_begin),
                                       int(n_end), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                                       _stream(stream)), "kvswap_project_keys")
+
+
+def kvswap_append_kv(shape: kvswap_shape, k_new, v_new, K, V, proj, meta, stream=None) -> bool:
+    """Appends one token's entries at row shape.n_ctx; True if that completed (and flushed) a group."""
+    flushed = ctypes.c_int32(0)
+    _check(load().kvswap_append_kv(ctypes.byref(shape), _ptr(k_new), _ptr(v_new), _ptr(K), _ptr(V), _ptr(proj),
+                                   _ptr(meta), ctypes.byref(flushed), _stream(stream)), "kvswap_append_kv")
+    return bool(flushed.value)
 
 
 def kvswap_score_select(shape, q, proj, meta, group_idx, n_selected, group_scores_opt, ws, stream=None) -> None:

@@ -153,6 +153,34 @@ static cudaError_t score_select_launch(const Problem& p, const Workspace& w, con
   return e;
 }
 
+int kvswap_append_kv(const kvswap_shape* shape, const void* k_new, const void* v_new, void* K, void* V,
+                     const float* proj, void* meta, int32_t* flushed_opt, void* cuda_stream) {
+  if (flushed_opt != nullptr) *flushed_opt = 0;
+  if (shape == nullptr) return KVSWAP_ERR_NULL;
+  // The store must say how many rows it has room for: dense strides would mean "exactly n_ctx".
+  if (shape->kv_stride_h == 0 || shape->meta_stride_h == 0) return KVSWAP_ERR_SHAPE;
+  if (shape->n_ctx >= (1 << 30)) return KVSWAP_ERR_SHAPE;
+  kvswap_shape grown = *shape;
+  grown.n_ctx = shape->n_ctx + 1;
+  Problem p;
+  int st = resolve(&grown, &p);
+  if (st != KVSWAP_OK) return st;
+  if (k_new == nullptr || v_new == nullptr || K == nullptr || V == nullptr || proj == nullptr || meta == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (misaligned(k_new) || misaligned(v_new) || misaligned(K) || misaligned(V) || misaligned(proj) || misaligned(meta))
+    return KVSWAP_ERR_ALIGN;
+  if (p.kv_sh < int64_t(p.N) * p.kv_sn || p.meta_sh < int64_t(p.N) * p.meta_sn) return KVSWAP_ERR_SHAPE;   // no room
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int n = p.N - 1;                                       // row of the new token
+  if (launch_append_rows(p, k_new, v_new, K, V, n, stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+  if (p.N % p.G == 0) {                                        // the new token completes a group: flush it
+    if (launch_project_keys(p, K, proj, meta, p.N - p.G, p.N, nullptr, nullptr, stream) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+    if (flushed_opt != nullptr) *flushed_opt = 1;
+  }
+  return KVSWAP_OK;
+}
+
 int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
                         int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
                         size_t ws_bytes, void* cuda_stream) {

@@ -48,6 +48,8 @@ void plan_sparse_decode(const Problem& p, Workspace* w);   // fills splits, head
 // `scratch` is the workspace region at off_adapter (project_keys_umma_scratch_bytes, may be NULL).
 cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta,
                                 int n_begin, int n_end, void* scratch, uint32_t* err, cudaStream_t st);
+cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* v_new, void* K, void* V, int n,
+                               cudaStream_t st);
 size_t project_keys_umma_scratch_bytes(const Problem& p);
 bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
                                   int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result);

@@ -315,15 +315,17 @@ cudaError_t dispatch_rc(const Problem& p, const void* K, const float* proj, void
   return cudaGetLastError();
 }
 
+constexpr int kMinTensorCoreTokens = 256;
+
 template <typename KV_T>
 cudaError_t dispatch_meta(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
-                          cudaStream_t st) {
+                          bool tensor_cores, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   if (p.meta_dtype == KVSWAP_F16) {
-    if (try_launch_mma<__half>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
+    if (tensor_cores && try_launch_mma<__half>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
     return dispatch_rc<KV_T, __half>(p, K, proj, meta, n_begin, n_end, st);
   }
-  if (try_launch_mma<float>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
+  if (tensor_cores && try_launch_mma<float>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
   return dispatch_rc<KV_T, float>(p, K, proj, meta, n_begin, n_end, st);
 }
 
@@ -332,11 +334,14 @@ cudaError_t dispatch_meta(const Problem& p, const void* K, const float* proj, vo
 cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
                                 int n_end, void* scratch, uint32_t* err, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
-  if (try_launch_project_keys_umma(p, K, proj, meta, n_begin, n_end, scratch, err, st, &e)) return e;
+  // A short token range (a flushed group during decoding) is not worth the tensor-core paths'
+  // set-up (adapter split, tensor maps, shared-memory-resident operand fragments).
+  const bool tensor_cores = n_end - n_begin >= kMinTensorCoreTokens;
+  if (tensor_cores && try_launch_project_keys_umma(p, K, proj, meta, n_begin, n_end, scratch, err, st, &e)) return e;
   switch (p.kv_dtype) {
-    case KVSWAP_F32: return dispatch_meta<float>(p, K, proj, meta, n_begin, n_end, st);
-    case KVSWAP_BF16: return dispatch_meta<__nv_bfloat16>(p, K, proj, meta, n_begin, n_end, st);
-    default: return dispatch_meta<__half>(p, K, proj, meta, n_begin, n_end, st);
+    case KVSWAP_F32: return dispatch_meta<float>(p, K, proj, meta, n_begin, n_end, tensor_cores, st);
+    case KVSWAP_BF16: return dispatch_meta<__nv_bfloat16>(p, K, proj, meta, n_begin, n_end, tensor_cores, st);
+    default: return dispatch_meta<__half>(p, K, proj, meta, n_begin, n_end, tensor_cores, st);
   }
 }
 

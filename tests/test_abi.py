@@ -105,6 +105,23 @@ def test_entry_points_reject_null_and_small_workspace_without_touching_the_gpu(l
     assert lib.kvswap_sparse_decode(ref, fake, fake, fake, fake, fake, fake, None, fake, 16, None) == 5
 
 
+def test_append_kv_validates_before_touching_the_gpu(lib):
+    fake = ctypes.c_void_p(4096)
+    flushed = ctypes.c_int32(7)
+    dense = good_shape()
+    assert lib.kvswap_append_kv(ctypes.byref(dense), fake, fake, fake, fake, fake, fake, ctypes.byref(flushed), None) == 2
+    assert flushed.value == 0
+    N, d, r = 1024, 64, 16
+    roomy = good_shape(kv_strides=(2 * (N + 8) * d, (N + 8) * d, d), meta_strides=((N + 8) * r, (N + 8) * r, r))
+    assert lib.kvswap_append_kv(ctypes.byref(roomy), None, fake, fake, fake, fake, fake, None, None) == 1
+    assert lib.kvswap_append_kv(ctypes.byref(roomy), ctypes.c_void_p(4100), fake, fake, fake, fake, fake, None, None) == 4
+    tight = good_shape(kv_strides=(2 * N * d, N * d, d), meta_strides=((N + 8) * r, (N + 8) * r, r))
+    assert lib.kvswap_append_kv(ctypes.byref(tight), fake, fake, fake, fake, fake, fake, None, None) == 2   # K/V full
+    tight_meta = good_shape(kv_strides=(2 * (N + 8) * d, (N + 8) * d, d), meta_strides=(N * r, N * r, r))
+    assert lib.kvswap_append_kv(ctypes.byref(tight_meta), fake, fake, fake, fake, fake, fake, None, None) == 2
+    assert lib.kvswap_append_kv(None, fake, fake, fake, fake, fake, fake, None, None) == 1
+
+
 def test_status_strings_and_version(lib):
     seen = {kv.status_string(i) for i in range(11)}
     assert len(seen) == 11 and "ok" in seen
