@@ -365,8 +365,42 @@ def run_ours(args, wl):
     e2e_ms = e0.elapsed_time(e1)
     clocks = sampler.stop(wall0, wall1) if sampler else None
 
+    # ---- growing context (Sec. 4.4.1): every step first appends one token per layer to the rolling buffer
+    # (a completed group is flushed into the compact cache), then decodes over the grown context.  The
+    # store's last rows serve as the spare rows, so the walk ends at the full length N. ------------------------
+    N, Hkv, d_, r_ = wl.n_ctx, wl.n_kv_heads, wl.head_dim, wl.rank
+    grow_steps = max(1, min(64, steps, N - 1))
+    cap = dict(kv_strides=(Hkv * N * d_, N * d_, d_), meta_strides=(meta_heads * N * r_, N * r_, r_))
+    grow_shapes = [rt.shape_for(wl, meta_heads, scope, n_ctx=n, **cap) for n in range(N - grow_steps, N + 1)]
+    kv_t = dw.K[0].dtype
+    k_new = torch.randn((L, wl.batch, Hkv, d_), device=dev).to(kv_t)
+    v_new = torch.randn((L, wl.batch, Hkv, d_), device=dev).to(kv_t)
+
+    def grow(t):
+        kv.kvswap_append_step(grow_shapes[t], layers, k_new, v_new)
+        kv.kvswap_decode_step(grow_shapes[t + 1], layers, dw.q_walk[t % n_walk], out, None, idx, nsel, ws, None)
+
+    for t in range(min(2, grow_steps)):
+        grow(t)
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    g0.record()
+    for t in range(grow_steps):
+        grow(t)
+    g1.record()
+    sync_all()
+    grow_ms = g0.elapsed_time(g1)
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for t in range(grow_steps):
+        kv.kvswap_append_step(grow_shapes[t], layers, k_new, v_new)
+    a1.record()
+    sync_all()
+    append_ms = a0.elapsed_time(a1)
+
     # ---- max over ranks ----------------------------------------------------------------------------
-    elapsed_ms, e2e_ms, look1_ms = shard.max_over_ranks([elapsed_ms, e2e_ms, look1_ms], device=dev)
+    elapsed_ms, e2e_ms, look1_ms, grow_ms, append_ms = shard.max_over_ranks(
+        [elapsed_ms, e2e_ms, look1_ms, grow_ms, append_ms], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -401,6 +435,10 @@ def run_ours(args, wl):
         "schedule": {"predictor_lookahead_layers": "unbounded",
                      "lookahead_1": {"value": world * 1e3 * n1 / look1_ms, "unit": UNIT, "steps": n1,
                                      "ms_per_step": look1_ms / n1}},
+        "growing_context": {"value": world * 1e3 * grow_steps / grow_ms, "unit": UNIT, "steps": grow_steps,
+                            "n_ctx": [N - grow_steps, N], "ms_per_step": grow_ms / grow_steps,
+                            "append_ms_per_step": append_ms / grow_steps,
+                            "flushes": sum(1 for n in range(N - grow_steps, N) if (n + 1) % wl.group_size == 0)},
         "e2e": {"value": world * 1e3 * e2e_steps / e2e_ms, "unit": UNIT, "h2d_bytes_per_step": q_bytes,
                 "d2h_bytes_per_step": out_bytes, "steps": e2e_steps},
         "gpu_launches": 5 * L * steps,

@@ -244,6 +244,17 @@ typedef struct {
 } kvswap_probe;
 
 /*
+ * kvswap_append_kv for every layer of a model at once: k_new, v_new [L, B, H_kv, d] kv_dtype
+ * (dense, device) join row N = shape->n_ctx of layers->K[l], layers->V[l] (one launch per 32
+ * layers); when that completes a group, each layer's compact-cache rows of the group are built.
+ * The tables are const-qualified for the read-only calls; this call WRITES the K, V and meta
+ * buffers they point to.  max_lookahead is ignored.  Same errors and capacity rule as
+ * kvswap_append_kv.
+ */
+int kvswap_append_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* k_new,
+                       const void* v_new, int32_t* flushed_opt, void* cuda_stream);
+
+/*
  * One decode step of the predictor + sparse attention (Sec. 4.4, decoding): for l = 0..L-1, in
  * order on `cuda_stream`, kvswap_score_select then kvswap_sparse_decode on layer l, with
  *   q          [L, B, H_q, d] q_dtype  (the same query scores and attends; device)

@@ -211,6 +211,8 @@ def _declare_step(lib):
     P, PL, PP = ctypes.POINTER(kvswap_shape), ctypes.POINTER(kvswap_layers), ctypes.POINTER(kvswap_probe)
     lib.kvswap_decode_step.restype = ctypes.c_int
     lib.kvswap_decode_step.argtypes = [P, PL, V, V, V, V, V, V, SZ, PP, V]
+    lib.kvswap_append_step.restype = ctypes.c_int
+    lib.kvswap_append_step.argtypes = [P, PL, V, V, ctypes.POINTER(ctypes.c_int32), V]
     lib.kvswap_decode_step_host.restype = ctypes.c_int
     lib.kvswap_decode_step_host.argtypes = [P, PL, V, V, V, V, V, V, V, SZ, V]
     lib._step_declared = True
@@ -223,6 +225,15 @@ def kvswap_decode_step(shape, layers, q, out, lse_opt, group_idx, n_selected, ws
                                   _ptr(group_idx), _ptr(n_selected), _ptr(ws), ws.numel() * ws.element_size(),
                                   None if probe_opt is None else ctypes.byref(probe_opt), _stream(stream)),
            "kvswap_decode_step")
+
+
+def kvswap_append_step(shape, layers, k_new, v_new, stream=None) -> bool:
+    """Appends one token per layer (k_new, v_new [L, B, H_kv, d]) at row shape.n_ctx; True if a group was flushed."""
+    lib = _declare_step(load())
+    flushed = ctypes.c_int32(0)
+    _check(lib.kvswap_append_step(ctypes.byref(shape), ctypes.byref(layers), _ptr(k_new), _ptr(v_new),
+                                  ctypes.byref(flushed), _stream(stream)), "kvswap_append_step")
+    return bool(flushed.value)
 
 
 def kvswap_decode_step_host(shape, layers, q_host, out_host, q_dev, out_dev, group_idx, n_selected, ws,

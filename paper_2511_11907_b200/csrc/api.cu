@@ -60,15 +60,20 @@ int resolve(const kvswap_shape* s, Problem* p) {
   p->NG = p->N / p->G;
   p->Mp = std::min(p->M, p->NG);
   p->Su = (p->Hm == 1) ? p->S : p->Hkv;
+  p->score_pitch = p->NG;
   return KVSWAP_OK;
 }
+
+// Rows of the workspace's group-score buffer are padded to whole 16-byte vectors (128 bytes), so
+// that the top-k kernel can load them as vectors whatever NG is.
+static int workspace_score_pitch(const Problem& p) { return (std::max(p.NG, 1) + 31) / 32 * 32; }
 
 void plan_workspace(const Problem& p, Workspace* w) {
   plan_sparse_decode(p, w);
 
   size_t off = 256;  // first 256 bytes reserved
   w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
-  w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * std::max(p.NG, 1));
+  w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * workspace_score_pitch(p));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
   w->off_adapter = off;  off += align256(project_keys_umma_scratch_bytes(p) + 1024);   // 1 KiB: tensor-map base alignment
   w->total = off;
@@ -141,40 +146,81 @@ static int check_score_select(const kvswap_shape* shape, const void* q, const fl
 }
 
 // The three launches of the predictor for one layer (arguments already checked).
-static cudaError_t score_select_launch(const Problem& p, const Workspace& w, const void* q, const float* proj,
+static cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, const void* q, const float* proj,
                                        const void* meta, int32_t* group_idx, int32_t* n_selected,
                                        float* group_scores_opt, void* ws, cudaStream_t stream) {
   char* base = static_cast<char*>(ws);
   float* uq = reinterpret_cast<float*>(base + w.off_uq);
   float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
+  Problem p = p_in;
+  p.score_pitch = group_scores_opt ? p.NG : workspace_score_pitch(p);     // a caller's buffer is dense [B, S, NG]
   cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
   if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
   if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
   return e;
 }
 
-int kvswap_append_kv(const kvswap_shape* shape, const void* k_new, const void* v_new, void* K, void* V,
-                     const float* proj, void* meta, int32_t* flushed_opt, void* cuda_stream) {
-  if (flushed_opt != nullptr) *flushed_opt = 0;
+// Checks shared by the append calls; on success `p` describes the grown context (N + 1 tokens).
+static int resolve_grown(const kvswap_shape* shape, Problem* p) {
   if (shape == nullptr) return KVSWAP_ERR_NULL;
   // The store must say how many rows it has room for: dense strides would mean "exactly n_ctx".
   if (shape->kv_stride_h == 0 || shape->meta_stride_h == 0) return KVSWAP_ERR_SHAPE;
   if (shape->n_ctx >= (1 << 30)) return KVSWAP_ERR_SHAPE;
   kvswap_shape grown = *shape;
   grown.n_ctx = shape->n_ctx + 1;
+  int st = resolve(&grown, p);
+  if (st != KVSWAP_OK) return st;
+  if (p->kv_sh < int64_t(p->N) * p->kv_sn || p->meta_sh < int64_t(p->N) * p->meta_sn) return KVSWAP_ERR_SHAPE;  // no room
+  return KVSWAP_OK;
+}
+
+int kvswap_append_kv(const kvswap_shape* shape, const void* k_new, const void* v_new, void* K, void* V,
+                     const float* proj, void* meta, int32_t* flushed_opt, void* cuda_stream) {
+  if (flushed_opt != nullptr) *flushed_opt = 0;
   Problem p;
-  int st = resolve(&grown, &p);
+  int st = resolve_grown(shape, &p);
   if (st != KVSWAP_OK) return st;
   if (k_new == nullptr || v_new == nullptr || K == nullptr || V == nullptr || proj == nullptr || meta == nullptr)
     return KVSWAP_ERR_NULL;
   if (misaligned(k_new) || misaligned(v_new) || misaligned(K) || misaligned(V) || misaligned(proj) || misaligned(meta))
     return KVSWAP_ERR_ALIGN;
-  if (p.kv_sh < int64_t(p.N) * p.kv_sn || p.meta_sh < int64_t(p.N) * p.meta_sn) return KVSWAP_ERR_SHAPE;   // no room
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const int n = p.N - 1;                                       // row of the new token
-  if (launch_append_rows(p, k_new, v_new, K, V, n, stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
+  if (launch_append_rows(p, k_new, v_new, &K, &V, 1, p.N - 1, stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
   if (p.N % p.G == 0) {                                        // the new token completes a group: flush it
     if (launch_project_keys(p, K, proj, meta, p.N - p.G, p.N, nullptr, nullptr, stream) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+    if (flushed_opt != nullptr) *flushed_opt = 1;
+  }
+  return KVSWAP_OK;
+}
+
+int kvswap_append_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* k_new, const void* v_new,
+                       int32_t* flushed_opt, void* cuda_stream) {
+  if (flushed_opt != nullptr) *flushed_opt = 0;
+  Problem p;
+  int st = resolve_grown(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  if (layers == nullptr || layers->K == nullptr || layers->V == nullptr || layers->meta == nullptr ||
+      layers->proj == nullptr || k_new == nullptr || v_new == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (layers->n_layers < 1) return KVSWAP_ERR_SHAPE;
+  if (misaligned(k_new) || misaligned(v_new)) return KVSWAP_ERR_ALIGN;
+  for (int l = 0; l < layers->n_layers; ++l) {
+    if (layers->K[l] == nullptr || layers->V[l] == nullptr || layers->meta[l] == nullptr || layers->proj[l] == nullptr)
+      return KVSWAP_ERR_NULL;
+    if (misaligned(layers->K[l]) || misaligned(layers->V[l]) || misaligned(layers->meta[l]) ||
+        misaligned(layers->proj[l]))
+      return KVSWAP_ERR_ALIGN;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // The tables are declared const for the read-only calls; this one writes the stores.
+  void* const* Ks = const_cast<void* const*>(layers->K);
+  void* const* Vs = const_cast<void* const*>(layers->V);
+  if (launch_append_rows(p, k_new, v_new, Ks, Vs, layers->n_layers, p.N - 1, stream) != cudaSuccess)
+    return KVSWAP_ERR_CUDA;
+  if (p.N % p.G == 0) {
+    if (launch_project_keys_layers(p, layers->K, layers->proj, const_cast<void* const*>(layers->meta),
+                                   layers->n_layers, p.N - p.G, p.N, stream) != cudaSuccess)
       return KVSWAP_ERR_CUDA;
     if (flushed_opt != nullptr) *flushed_opt = 1;
   }

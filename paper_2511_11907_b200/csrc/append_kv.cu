@@ -5,40 +5,64 @@
 // one row copy per (sequence, KV head) for K and for V; the "flush" of a completed group leaves the
 // rows where they are and only builds the group's rows of the compact cache (project_keys over
 // the group's token range).
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace kvswap {
 namespace {
 
-// One CTA per (sequence, KV head): the first half of the threads copies the K row, the second half
-// the V row, 16 bytes per thread.
+constexpr int kMaxAppendLayers = 32;
+
+// Stores of the layers one launch serves (blockIdx.y = layer).
+struct StoreTable {
+  unsigned char* K[kMaxAppendLayers];
+  unsigned char* V[kMaxAppendLayers];
+};
+
+// One CTA per (sequence, KV head, layer): the first half of the threads copies the K row, the
+// second half the V row, 16 bytes per thread.  k_new, v_new: [layers, B, H_kv, d].
 __global__ void append_rows_kernel(const unsigned char* __restrict__ k_new, const unsigned char* __restrict__ v_new,
-                                   unsigned char* __restrict__ K, unsigned char* __restrict__ V, int Hkv, int row_bytes,
-                                   int64_t sb_bytes, int64_t sh_bytes, int64_t row_offset_bytes) {
-  const int bg = blockIdx.x, b = bg / Hkv, g = bg % Hkv;
+                                   const StoreTable stores, int Hkv, int row_bytes, int64_t sb_bytes, int64_t sh_bytes,
+                                   int64_t row_offset_bytes) {
+  const int bg = blockIdx.x, b = bg / Hkv, g = bg % Hkv, layer = blockIdx.y;
   const int pieces = row_bytes / 16;
   const int t = threadIdx.x;
   const bool is_v = t >= pieces;
   const int piece = is_v ? t - pieces : t;
   if (piece >= pieces) return;
-  const unsigned char* src = (is_v ? v_new : k_new) + int64_t(bg) * row_bytes + piece * 16;
-  unsigned char* dst = (is_v ? V : K) + int64_t(b) * sb_bytes + int64_t(g) * sh_bytes + row_offset_bytes + piece * 16;
+  const int64_t src_off = (int64_t(layer) * gridDim.x + bg) * row_bytes + piece * 16;
+  const unsigned char* src = (is_v ? v_new : k_new) + src_off;
+  unsigned char* dst = (is_v ? stores.V[layer] : stores.K[layer]) + int64_t(b) * sb_bytes + int64_t(g) * sh_bytes +
+                       row_offset_bytes + piece * 16;
   *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
 }
 
 }  // namespace
 
-// Writes k_new, v_new [B, H_kv, d] to token row `n` of K and V (strides of `p`).
-cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* v_new, void* K, void* V, int n,
-                               cudaStream_t st) {
+// Writes k_new, v_new [n_layers, B, H_kv, d] to token row `n` of each layer's K and V (strides of
+// `p`), kMaxAppendLayers layers per launch.
+cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* v_new, void* const* K, void* const* V,
+                               int n_layers, int n, cudaStream_t st) {
   const int e = (p.kv_dtype == KVSWAP_F32) ? 4 : 2;
   const int row_bytes = p.d * e;                     // 128 .. 512, a multiple of 16
   const int threads = 2 * (row_bytes / 16);
-  append_rows_kernel<<<p.B * p.Hkv, threads, 0, st>>>(
-      static_cast<const unsigned char*>(k_new), static_cast<const unsigned char*>(v_new),
-      static_cast<unsigned char*>(K), static_cast<unsigned char*>(V), p.Hkv, row_bytes, p.kv_sb * e, p.kv_sh * e,
-      int64_t(n) * p.kv_sn * e);
-  return cudaGetLastError();
+  const int64_t layer_bytes = int64_t(p.B) * p.Hkv * row_bytes;
+  for (int l0 = 0; l0 < n_layers; l0 += kMaxAppendLayers) {
+    const int count = std::min(kMaxAppendLayers, n_layers - l0);
+    StoreTable stores = {};
+    for (int l = 0; l < count; ++l) {
+      stores.K[l] = static_cast<unsigned char*>(K[l0 + l]);
+      stores.V[l] = static_cast<unsigned char*>(V[l0 + l]);
+    }
+    append_rows_kernel<<<dim3(p.B * p.Hkv, count), threads, 0, st>>>(
+        static_cast<const unsigned char*>(k_new) + l0 * layer_bytes,
+        static_cast<const unsigned char*>(v_new) + l0 * layer_bytes, stores, p.Hkv, row_bytes, p.kv_sb * e,
+        p.kv_sh * e, int64_t(n) * p.kv_sn * e);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace kvswap

@@ -26,6 +26,7 @@ struct Problem {
   int NG;    // complete groups
   int Mp;    // min(M, NG)
   int Su;    // rows of the low-rank query buffer per sequence (see score_pool.cu)
+  int score_pitch;   // floats between rows of the group-score buffer: NG in a caller's buffer, padded in the workspace
 };
 
 // Partition of the caller's workspace (byte offsets, each 256-byte aligned).
@@ -48,8 +49,10 @@ void plan_sparse_decode(const Problem& p, Workspace* w);   // fills splits, head
 // `scratch` is the workspace region at off_adapter (project_keys_umma_scratch_bytes, may be NULL).
 cudaError_t launch_project_keys(const Problem& p, const void* K, const float* proj, void* meta,
                                 int n_begin, int n_end, void* scratch, uint32_t* err, cudaStream_t st);
-cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* v_new, void* K, void* V, int n,
-                               cudaStream_t st);
+cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* v_new, void* const* K, void* const* V,
+                               int n_layers, int n, cudaStream_t st);
+cudaError_t launch_project_keys_layers(const Problem& p, const void* const* K, const float* const* proj,
+                                       void* const* meta, int n_layers, int n_begin, int n_end, cudaStream_t st);
 size_t project_keys_umma_scratch_bytes(const Problem& p);
 bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
                                   int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result);

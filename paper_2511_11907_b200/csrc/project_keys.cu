@@ -21,18 +21,29 @@ constexpr int kTok = 64;      // tokens per CTA
 constexpr int kChunk = 32;    // contraction chunk
 constexpr int kThreads = 256;
 
+// Buffers of the layers one launch serves (a flushed group is projected for all layers at once).
+constexpr int kMaxProjectLayers = 32;
+struct ProjectTable {
+  const void* K[kMaxProjectLayers];
+  const float* proj[kMaxProjectLayers];
+  void* meta[kMaxProjectLayers];
+};
+
 template <typename KV_T, typename META_T, int RC>   // RC = ceil(r / 32) output columns per lane
 __global__ void __launch_bounds__(kThreads)
-project_keys_kernel(Problem p, const KV_T* __restrict__ K, const float* __restrict__ proj,
-                    META_T* __restrict__ meta, int n_begin, int n_end) {
+project_keys_kernel(Problem p, const ProjectTable tab, int tiles, int n_begin, int n_end) {
   __shared__ float Ks[kTok][kChunk + 1];
   __shared__ float Ps[kChunk][32 * RC];
 
+  const int layer = blockIdx.x / tiles;            // blockIdx.x = layer * tiles + token tile
+  const KV_T* __restrict__ K = static_cast<const KV_T*>(tab.K[layer]);
+  const float* __restrict__ proj = tab.proj[layer];
+  META_T* __restrict__ meta = static_cast<META_T*>(tab.meta[layer]);
   const int b = blockIdx.y;
   const int head_out = blockIdx.z;                 // per-head layout: the KV head; joint: 0
   const int g_first = (p.Hm == 1) ? 0 : head_out;
   const int g_count = (p.Hm == 1) ? p.Hkv : 1;
-  const int n0 = n_begin + blockIdx.x * kTok;
+  const int n0 = n_begin + (blockIdx.x % tiles) * kTok;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   float acc[8][RC];
@@ -302,17 +313,32 @@ bool try_launch_mma(const Problem& p, const void* K, const float* proj, void* me
 }
 
 template <typename KV_T, typename META_T>
-cudaError_t dispatch_rc(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
+cudaError_t dispatch_rc(const Problem& p, const ProjectTable& tab, int n_layers, int n_begin, int n_end,
                         cudaStream_t st) {
-  dim3 grid((n_end - n_begin + kTok - 1) / kTok, p.B, p.Hm);
-  const KV_T* Kt = static_cast<const KV_T*>(K);
-  META_T* Mt = static_cast<META_T*>(meta);
+  const int tiles = (n_end - n_begin + kTok - 1) / kTok;
+  dim3 grid(tiles * n_layers, p.B, p.Hm);
   const int rc = (p.r + 31) / 32;
-  if (rc <= 1) project_keys_kernel<KV_T, META_T, 1><<<grid, kThreads, 0, st>>>(p, Kt, proj, Mt, n_begin, n_end);
-  else if (rc <= 2) project_keys_kernel<KV_T, META_T, 2><<<grid, kThreads, 0, st>>>(p, Kt, proj, Mt, n_begin, n_end);
-  else if (rc <= 4) project_keys_kernel<KV_T, META_T, 4><<<grid, kThreads, 0, st>>>(p, Kt, proj, Mt, n_begin, n_end);
-  else project_keys_kernel<KV_T, META_T, 8><<<grid, kThreads, 0, st>>>(p, Kt, proj, Mt, n_begin, n_end);
+  if (rc <= 1) project_keys_kernel<KV_T, META_T, 1><<<grid, kThreads, 0, st>>>(p, tab, tiles, n_begin, n_end);
+  else if (rc <= 2) project_keys_kernel<KV_T, META_T, 2><<<grid, kThreads, 0, st>>>(p, tab, tiles, n_begin, n_end);
+  else if (rc <= 4) project_keys_kernel<KV_T, META_T, 4><<<grid, kThreads, 0, st>>>(p, tab, tiles, n_begin, n_end);
+  else project_keys_kernel<KV_T, META_T, 8><<<grid, kThreads, 0, st>>>(p, tab, tiles, n_begin, n_end);
   return cudaGetLastError();
+}
+
+template <typename KV_T>
+cudaError_t dispatch_rc_meta(const Problem& p, const ProjectTable& tab, int n_layers, int n_begin, int n_end,
+                             cudaStream_t st) {
+  if (p.meta_dtype == KVSWAP_F16) return dispatch_rc<KV_T, __half>(p, tab, n_layers, n_begin, n_end, st);
+  return dispatch_rc<KV_T, float>(p, tab, n_layers, n_begin, n_end, st);
+}
+
+cudaError_t dispatch_table(const Problem& p, const ProjectTable& tab, int n_layers, int n_begin, int n_end,
+                           cudaStream_t st) {
+  switch (p.kv_dtype) {
+    case KVSWAP_F32: return dispatch_rc_meta<float>(p, tab, n_layers, n_begin, n_end, st);
+    case KVSWAP_BF16: return dispatch_rc_meta<__nv_bfloat16>(p, tab, n_layers, n_begin, n_end, st);
+    default: return dispatch_rc_meta<__half>(p, tab, n_layers, n_begin, n_end, st);
+  }
 }
 
 constexpr int kMinTensorCoreTokens = 256;
@@ -321,12 +347,16 @@ template <typename KV_T>
 cudaError_t dispatch_meta(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
                           bool tensor_cores, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
-  if (p.meta_dtype == KVSWAP_F16) {
-    if (tensor_cores && try_launch_mma<__half>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
-    return dispatch_rc<KV_T, __half>(p, K, proj, meta, n_begin, n_end, st);
+  if (tensor_cores) {
+    if (p.meta_dtype == KVSWAP_F16) {
+      if (try_launch_mma<__half>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
+    } else if (try_launch_mma<float>(p, K, proj, meta, n_begin, n_end, st, &e)) {
+      return e;
+    }
   }
-  if (tensor_cores && try_launch_mma<float>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
-  return dispatch_rc<KV_T, float>(p, K, proj, meta, n_begin, n_end, st);
+  ProjectTable tab = {};
+  tab.K[0] = K; tab.proj[0] = proj; tab.meta[0] = meta;
+  return dispatch_rc_meta<KV_T>(p, tab, 1, n_begin, n_end, st);
 }
 
 }  // namespace
@@ -343,6 +373,20 @@ cudaError_t launch_project_keys(const Problem& p, const void* K, const float* pr
     case KVSWAP_BF16: return dispatch_meta<__nv_bfloat16>(p, K, proj, meta, n_begin, n_end, tensor_cores, st);
     default: return dispatch_meta<__half>(p, K, proj, meta, n_begin, n_end, tensor_cores, st);
   }
+}
+
+// The same token range of several layers (a group flushed during decoding) on the fp32 path, up
+// to kMaxProjectLayers layers per launch.
+cudaError_t launch_project_keys_layers(const Problem& p, const void* const* K, const float* const* proj,
+                                       void* const* meta, int n_layers, int n_begin, int n_end, cudaStream_t st) {
+  for (int l0 = 0; l0 < n_layers; l0 += kMaxProjectLayers) {
+    const int count = std::min(kMaxProjectLayers, n_layers - l0);
+    ProjectTable tab = {};
+    for (int l = 0; l < count; ++l) { tab.K[l] = K[l0 + l]; tab.proj[l] = proj[l0 + l]; tab.meta[l] = meta[l0 + l]; }
+    cudaError_t e = dispatch_table(p, tab, count, n_begin, n_end, st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace kvswap

@@ -298,7 +298,7 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
       const int ns = (p.Hm == 1) ? min(NS, p.S - s0) : 1;
       for (int i = lane; i < ns * ngt; i += 32) {
         const int s = i / ngt, gi = i - s * ngt;
-        scores[(int64_t(b) * p.S + s0 + s) * p.NG + g0 + gi] = out[s * kOutStride + gi];
+        scores[(int64_t(b) * p.S + s0 + s) * p.score_pitch + g0 + gi] = out[s * kOutStride + gi];
       }
     }
     __syncwarp();                                   // stage and outbuf are free again
@@ -448,7 +448,7 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
       }
       const int s0 = (p.Hm == 1) ? sub * NS : hm;
       ns_cur = (p.Hm == 1) ? min(NS, p.S - s0) : 1;
-      out_row0 = scores + (int64_t(b) * p.S + s0) * p.NG;
+      out_row0 = scores + (int64_t(b) * p.S + s0) * p.score_pitch;
     }
     if (++c_tile == tiles_per_row) { c_tile = 0; ++c_rest; }
     if (!__all_sync(kFull, mbar_wait(smem_addr(&ctl->full[warp * kDepth + stage]), phase))) { timed_out = true; break; }
@@ -499,12 +499,12 @@ score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __r
         const int sh = 5 - g_shift;
         for (int i = lane; i < (ns_cur << sh); i += 32) {
           const int s = i >> sh, gi = i & ((1 << sh) - 1);
-          dst[int64_t(s) * p.NG + gi] = out[s * kOutStride + gi];
+          dst[int64_t(s) * p.score_pitch + gi] = out[s * kOutStride + gi];
         }
       } else {
         for (int i = lane; i < ns_cur * ngt; i += 32) {
           const int s = i / ngt, gi = i - s * ngt;
-          dst[int64_t(s) * p.NG + gi] = out[s * kOutStride + gi];
+          dst[int64_t(s) * p.score_pitch + gi] = out[s * kOutStride + gi];
         }
       }
     }
@@ -593,7 +593,7 @@ score_pool_kernel(Problem p, const float* __restrict__ uq, const META_T* __restr
     const float* s = sc + k * tile_tok + gi * p.G;
     float m = s[0];
     for (int t = 1; t < p.G; ++t) m = fmaxf(m, s[t]);
-    scores[(int64_t(b) * p.S + out0 + k) * p.NG + grp0 + gi] = m;
+    scores[(int64_t(b) * p.S + out0 + k) * p.score_pitch + grp0 + gi] = m;
   }
 }
 

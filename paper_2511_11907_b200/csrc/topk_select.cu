@@ -60,7 +60,7 @@ topk_select_kernel(Problem p, const float* __restrict__ scores, int32_t* __restr
   pdl_wait();
   pdl_trigger();
   const int prob = blockIdx.x;                 // b * S + s
-  const float* R = scores + int64_t(prob) * p.NG;
+  const float* R = scores + int64_t(prob) * p.score_pitch;
   int32_t* out = group_idx + int64_t(prob) * p.M;
   const int NG = p.NG, Mp = p.Mp;
 
@@ -164,7 +164,7 @@ topk_select_regs_kernel(Problem p, const float* __restrict__ scores, int32_t* __
   for (int i = threadIdx.x; i < kBins; i += kThreads) hist[i] = 0;
   pdl_wait();
   pdl_trigger();
-  const float* R = scores + int64_t(prob) * NG;
+  const float* R = scores + int64_t(prob) * p.score_pitch;
   int32_t* out = group_idx + int64_t(prob) * p.M;
 
   if (threadIdx.x == 0) n_selected[prob] = Mp;
@@ -179,13 +179,15 @@ topk_select_regs_kernel(Problem p, const float* __restrict__ scores, int32_t* __
   const int i0 = int(threadIdx.x) * KPT;
   uint32_t key[KPT];
   if constexpr (KPT >= 4) {
-    if ((NG & 3) == 0) {
+    if ((p.score_pitch & 3) == 0) {              // rows start 16-byte aligned and are padded to whole vectors
 #pragma unroll
       for (int v = 0; v < KPT / 4; ++v) {
         if (i0 + 4 * v < NG) {
           const float4 f = *reinterpret_cast<const float4*>(R + i0 + 4 * v);
-          key[4 * v] = score_key(f.x); key[4 * v + 1] = score_key(f.y);
-          key[4 * v + 2] = score_key(f.z); key[4 * v + 3] = score_key(f.w);
+          key[4 * v] = score_key(f.x);
+          key[4 * v + 1] = (i0 + 4 * v + 1 < NG) ? score_key(f.y) : 0u;      // row padding, never a key
+          key[4 * v + 2] = (i0 + 4 * v + 2 < NG) ? score_key(f.z) : 0u;
+          key[4 * v + 3] = (i0 + 4 * v + 3 < NG) ? score_key(f.w) : 0u;
         } else {
           key[4 * v] = key[4 * v + 1] = key[4 * v + 2] = key[4 * v + 3] = 0u;
         }

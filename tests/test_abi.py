@@ -120,6 +120,15 @@ def test_append_kv_validates_before_touching_the_gpu(lib):
     tight_meta = good_shape(kv_strides=(2 * (N + 8) * d, (N + 8) * d, d), meta_strides=(N * r, N * r, r))
     assert lib.kvswap_append_kv(ctypes.byref(tight_meta), fake, fake, fake, fake, fake, fake, None, None) == 2
     assert lib.kvswap_append_kv(None, fake, fake, fake, fake, fake, fake, None, None) == 1
+    kv._declare_step(lib)
+    tab = (ctypes.c_void_p * 1)(4096)
+    ptab = ctypes.cast(tab, ctypes.POINTER(ctypes.c_void_p))
+    one = kv.kvswap_layers(1, 0, ptab, ptab, ptab, ptab)
+    assert lib.kvswap_append_step(ctypes.byref(dense), ctypes.byref(one), fake, fake, None, None) == 2
+    assert lib.kvswap_append_step(ctypes.byref(roomy), None, fake, fake, None, None) == 1
+    assert lib.kvswap_append_step(ctypes.byref(roomy), ctypes.byref(one), None, fake, None, None) == 1
+    none = kv.kvswap_layers(0, 0, ptab, ptab, ptab, ptab)
+    assert lib.kvswap_append_step(ctypes.byref(roomy), ctypes.byref(none), fake, fake, None, None) == 2
 
 
 def test_status_strings_and_version(lib):

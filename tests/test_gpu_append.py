@@ -121,6 +121,33 @@ def test_context_shorter_than_one_group_at_the_start():
     _grow_and_check(wl, 1, 1, KV, check_at={2, 3, 4, 5, 8, 11})
 
 
+def test_append_step_over_many_layers_equals_per_layer_appends():
+    """35 layers (two launches of the row copy), three tokens, the last one completing a group."""
+    wl = W.CONFIGS[3].reduced("cfg3-thin", layers=35, batch=2, n_ctx=8 * 5, n_q_heads=8, n_kv_heads=2, calib_rows=256)
+    L, B, Hkv, d, r, G = wl.layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.rank, wl.group_size
+    cap, n0 = wl.n_ctx, 8 * 4 + 5
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    mk = lambda *shape: torch.randn(shape, generator=gen, device="cuda").to(torch.bfloat16)
+    Ka, Va = [mk(B, Hkv, cap, d) for _ in range(L)], [mk(B, Hkv, cap, d) for _ in range(L)]
+    Kb, Vb = [t.clone() for t in Ka], [t.clone() for t in Va]
+    proj = [torch.randn((Hkv, d, r), generator=gen, device="cuda") for _ in range(L)]
+    meta_a = [torch.full((B, 1, cap, r), float("nan"), dtype=torch.float16, device="cuda") for _ in range(L)]
+    meta_b = [t.clone() for t in meta_a]
+    strides = dict(kv_strides=(Hkv * cap * d, cap * d, d), meta_strides=(cap * r, cap * r, r))
+    tables = kv.make_layers(Kb, Vb, meta_b, proj)
+    for n in range(n0, n0 + 3):
+        sh = rt.shape_for(wl, 1, KV, n_ctx=n, **strides)
+        k_new, v_new = mk(L, B, Hkv, d), mk(L, B, Hkv, d)
+        flushed_a = [kv.kvswap_append_kv(sh, k_new[l], v_new[l], Ka[l], Va[l], proj[l], meta_a[l]) for l in range(L)]
+        flushed_b = kv.kvswap_append_step(sh, tables, k_new, v_new)
+        assert all(f == flushed_b for f in flushed_a) and flushed_b == ((n + 1) % G == 0)
+    torch.cuda.synchronize()
+    for l in range(L):
+        assert torch.equal(Ka[l], Kb[l]) and torch.equal(Va[l], Vb[l])
+        assert torch.equal(meta_a[l].view(torch.int16), meta_b[l].view(torch.int16))
+        assert torch.isfinite(meta_b[l][:, :, 8 * 4:8 * 5].float()).all() and torch.isnan(meta_b[l][:, :, :8 * 4].float()).all()
+
+
 def test_append_refuses_a_store_without_room():
     wl = W.CONFIGS[1].reduced("cfg1-full", batch=1, n_ctx=64)
     B, Hkv, N, d, r = wl.batch, wl.n_kv_heads, wl.n_ctx, wl.head_dim, wl.rank
