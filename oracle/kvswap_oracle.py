@@ -177,7 +177,7 @@ def attend(q, K, V, idx, G, scope="kv_head", return_probs=False):
 
 
 # ------------------------------------------------------------------------------------------
-# O7  New KV entries: rolling buffer, flush of a completed group                 (Sec. 4.4.1)
+# O8  New KV entries: rolling buffer, flush of a completed group                 (Sec. 4.4.1)
 # ------------------------------------------------------------------------------------------
 def append_kv(K, V, meta, k_new, v_new, proj, G, meta_dtype="f16"):
     """One generated token joins the cache.  Its entries k_new, v_new [B, H_kv, d] are appended to

@@ -441,7 +441,7 @@ def test_pins_detect_planted_mistakes(monkeypatch):
 
 
 # ------------------------------------------------------------------------------------------
-# O7  rolling-buffer append and group flush (Sec. 4.4.1)
+# O8  rolling-buffer append and group flush (Sec. 4.4.1)
 # ------------------------------------------------------------------------------------------
 def _grow(K0, V0, k_rows, v_rows, proj, G, meta_heads, meta_dtype="f64"):
     """Start from a context of K0.shape[2] tokens and append k_rows[t], v_rows[t] one by one."""
