@@ -197,3 +197,53 @@ def append_kv(K, V, meta, k_new, v_new, proj, G, meta_dtype="f16"):
         meta = np.concatenate([meta, rows.astype(meta.dtype)], axis=2)
     return K2, V2, meta, flushed
 
+
+# ------------------------------------------------------------------------------------------
+# O9  Reuse buffer: slots, slot table, FIFO replacement                          (Sec. 4.4.2)
+# ------------------------------------------------------------------------------------------
+def reuse_step(slot_group, head, selected):
+    """One prediction step of one reuse buffer (one sequence and selection scope).
+
+    slot_group[c] is the group id held by slot c (-1: empty) -- the paper's slot table; `head` is
+    the FIFO position: slots are filled in the order 0, 1, .., C-1, 0, .., so the slot at `head`
+    holds the group that was loaded longest ago.  `selected` lists the groups the predictor chose
+    for this step (distinct; entries < 0 mean "no group" and get slot -1).  In list order: a group
+    found in the slot table is a hit and keeps its slot; any other group is loaded into the next
+    slot in FIFO order, replacing what was there.  A slot that serves this step (a hit, or a
+    group loaded earlier in the same step) is passed over by the FIFO position, since the
+    attention of this step still reads it.
+
+    Returns (slots, loads, slot_group', head'): slots[i] the slot serving selected[i]; loads the
+    (group, slot) pairs fetched from the slow tier, in list order."""
+    table = [int(x) for x in slot_group]
+    C = len(table)
+    groups = [int(j) for j in selected if j >= 0]
+    if len(set(groups)) != len(groups):
+        raise ValueError("selected groups must be distinct")
+    if len(groups) > C:
+        raise ValueError("the reuse buffer must hold at least the groups of one step")
+    wanted = set(groups)
+    where = {g: c for c, g in enumerate(table) if g >= 0}
+    busy = {where[g] for g in groups if g in where}          # slots of this step's hits
+    slots, loads = [], []
+    for j in selected:
+        j = int(j)
+        if j < 0:
+            slots.append(-1)
+        elif j in where:
+            slots.append(where[j])
+        else:
+            while head in busy:
+                head = (head + 1) % C
+            old = table[head]
+            if old >= 0:
+                del where[old]
+            table[head] = j
+            where[j] = head
+            busy.add(head)
+            slots.append(head)
+            loads.append((j, head))
+            head = (head + 1) % C
+    assert all(table[where[g]] == g for g in wanted)
+    return slots, loads, table, head
+

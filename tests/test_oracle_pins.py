@@ -554,3 +554,112 @@ def test_planted_mistakes_in_append_are_caught(monkeypatch):
     assert fails(test_appended_token_is_attended_at_once_and_ranked_only_after_its_group_completes)
     monkeypatch.setattr(O, "append_kv", real)
 
+
+# ------------------------------------------------------------------------------------------
+# O9  reuse buffer (Sec. 4.4.2)
+# ------------------------------------------------------------------------------------------
+def test_reuse_buffer_hand_worked_fifo_trace():
+    """Four slots; every table below was written out by hand from the FIFO rule."""
+    table, head = [-1, -1, -1, -1], 0
+    slots, loads, table, head = O.reuse_step(table, head, [5, 9, 2])
+    assert (slots, loads, table, head) == ([0, 1, 2], [(5, 0), (9, 1), (2, 2)], [5, 9, 2, -1], 3)
+    slots, loads, table, head = O.reuse_step(table, head, [2, 7, 9])            # 2 and 9 hit, 7 takes the empty slot
+    assert (slots, loads, table, head) == ([2, 3, 1], [(7, 3)], [5, 9, 2, 7], 0)
+    slots, loads, table, head = O.reuse_step(table, head, [9, 4, 6])            # 5 is oldest; slot 1 (9) serves this step
+    assert (slots, loads, table, head) == ([1, 0, 2], [(4, 0), (6, 2)], [4, 9, 6, 7], 3)
+    slots, loads, table, head = O.reuse_step(table, head, [-1, 7, 3, -1])       # no-group entries; 7 hits at the head
+    assert (slots, loads, table, head) == ([-1, 3, 0, -1], [(3, 0)], [3, 9, 6, 7], 1)
+    slots, loads, table, head = O.reuse_step(table, head, [])
+    assert (slots, loads, table, head) == ([], [], [3, 9, 6, 7], 1)
+    slots, loads, table, head = O.reuse_step(table, head, [9])                  # a hit does not renew the slot's age
+    assert (slots, loads, table, head) == ([1], [], [3, 9, 6, 7], 1)
+    slots, loads, table, head = O.reuse_step(table, head, [8])                  # FIFO, not LRU: 9 goes although just used
+    assert (slots, loads, table, head) == ([1], [(8, 1)], [3, 8, 6, 7], 2)
+
+
+def test_reuse_buffer_against_a_queue_model_when_nothing_is_passed_over():
+    """With steps whose groups are all new (no hit can sit at the head) the buffer is a plain
+    FIFO queue of the last C loaded groups: compare with collections.deque."""
+    import collections
+    rng = np.random.default_rng(2)
+    C = 7
+    table, head = [-1] * C, 0
+    queue = collections.deque(maxlen=C)
+    fresh = iter(rng.permutation(1000))
+    for _ in range(40):
+        step = [int(next(fresh)) for _ in range(int(rng.integers(0, C + 1)))]
+        slots, loads, table, head = O.reuse_step(table, head, step)
+        queue.extend(step)
+        assert [g for g, _ in loads] == step and sorted(g for g in table if g >= 0) == sorted(queue)
+        assert [table[c] for c in slots] == step
+
+
+def test_reuse_buffer_invariants_on_random_walks():
+    """Random overlapping selections: every selected group is served by a slot that holds it, hits
+    keep their slot and cost no load, loads = misses, slots are never shared, and the buffer
+    only ever holds groups that were selected at some step."""
+    rng = np.random.default_rng(4)
+    C, NG, M = 12, 40, 8
+    table, head = [-1] * C, 0
+    prev = rng.choice(NG, size=M, replace=False)
+    ever = set()
+    for _ in range(200):
+        keep = rng.random(M) < 0.7
+        pool = np.setdiff1d(np.arange(NG), prev)
+        cur = np.where(keep, prev, rng.choice(pool, size=M, replace=False))
+        cur = np.array(list(dict.fromkeys(cur.tolist())))               # distinct, order kept
+        before = {g: c for c, g in enumerate(table) if g >= 0}
+        slots, loads, table, head = O.reuse_step(table, head, cur)
+        ever |= set(cur.tolist())
+        assert [table[c] for c in slots] == cur.tolist() and len(set(slots)) == len(slots)
+        hits = [g for g in cur.tolist() if g in before]
+        assert all(slots[cur.tolist().index(g)] == before[g] for g in hits)
+        assert sorted(g for g, _ in loads) == sorted(set(cur.tolist()) - set(before))
+        held = [g for g in table if g >= 0]
+        assert len(set(held)) == len(held) and set(held) <= ever and 0 <= head < C
+        prev = cur if len(cur) == M else rng.choice(NG, size=M, replace=False)
+
+
+def test_reuse_buffer_rejects_what_it_cannot_serve():
+    with pytest.raises(ValueError):
+        O.reuse_step([-1, -1], 0, [1, 2, 3])
+    with pytest.raises(ValueError):
+        O.reuse_step([-1, -1, -1], 0, [4, 4])
+
+
+def test_planted_mistakes_in_the_reuse_buffer_are_caught(monkeypatch):
+    real = O.reuse_step
+
+    def fails(test):
+        try:
+            test()
+        except (AssertionError, KeyError, ValueError):
+            return True
+        return False
+
+    def evicts_a_hit(slot_group, head, selected):                     # does not pass over busy slots
+        table = [int(x) for x in slot_group]
+        C = len(table)
+        slots, loads = [], []
+        for j in selected:
+            if j < 0:
+                slots.append(-1)
+            elif j in table:
+                slots.append(table.index(j))
+            else:
+                table[head] = int(j); slots.append(head); loads.append((int(j), head)); head = (head + 1) % C
+        return slots, loads, table, head
+    monkeypatch.setattr(O, "reuse_step", evicts_a_hit)
+    assert fails(test_reuse_buffer_hand_worked_fifo_trace)
+    assert fails(test_reuse_buffer_invariants_on_random_walks)
+
+    def lru_instead_of_fifo(slot_group, head, selected):              # a hit renews the slot's age
+        slots, loads, table, head2 = real(slot_group, head, selected)
+        hit_slots = [c for c, j in zip(slots, selected) if j >= 0 and (int(j), c) not in loads]
+        if hit_slots and not loads:
+            head2 = (max(hit_slots) + 1) % len(table)
+        return slots, loads, table, head2
+    monkeypatch.setattr(O, "reuse_step", lru_instead_of_fifo)
+    assert fails(test_reuse_buffer_hand_worked_fifo_trace)
+    monkeypatch.setattr(O, "reuse_step", real)
+
