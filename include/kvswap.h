@@ -244,6 +244,47 @@ typedef struct {
 } kvswap_probe;
 
 /*
+ * Reuse buffer (Sec. 4.4.2): n_slots slots per (sequence, selection scope), each holding the K/V
+ * rows of one group, in front of a slower tier that holds the whole cache (any memory the GPU can
+ * read: device memory, pinned host memory).  A slot table records the group in each slot; a
+ * selected group found there is a hit and is attended from its slot; any other is a miss: it
+ * takes the next slot in FIFO order (slots are filled in the order 0, 1, .., n_slots-1, 0, ..),
+ * passing over slots that serve the current step, and is fetched from the slow tier.
+ *
+ *   state       caller-owned device memory, kvswap_reuse_state_bytes(shape, n_slots, max_groups)
+ *               bytes, one per layer; kvswap_reuse_init empties every slot.  max_groups bounds
+ *               the group ids that will ever be looked up (floor(N_max / G)).
+ *   reuse store K_reuse, V_reuse [B, H_kv, (n_slots + 1) * G, d] kv_dtype, dense: slot c is rows
+ *               [c G, c G + G); the last G rows are room for the rolling buffer (the caller keeps
+ *               the N mod G newest tokens there).  With the per-KV-head scope head g's rows follow
+ *               head g's slot table; with the all-heads scope one table serves every head.
+ *
+ * kvswap_reuse_lookup takes a step's selection (group_idx [B, S, M], n_selected [B, S], as written
+ * by kvswap_score_select; entries must be distinct, entries outside [0, floor(n_ctx / G)) are "no
+ * group") and writes slot_idx [B, S, M] (the slot serving each entry, -1 for "no group"), the
+ * misses in list order as miss_group / miss_slot [B, S, M] (-1 beyond the count) and n_miss
+ * [B, S]; the slot table is updated.  kvswap_reuse_fill copies each missed group's G rows of K and
+ * V (of the scope's heads) from the slow tier, described by `shape`'s kv strides, into its slot.
+ * The step's attention is then kvswap_sparse_decode over the reuse store: K = K_reuse, V = V_reuse,
+ * group_idx = slot_idx, a shape with n_ctx = n_slots * G + (N mod G) and the reuse store's strides.
+ * Hits / (hits + misses) is the paper's reuse rate.
+ *
+ * Limits: n_slots >= M (else KVSWAP_ERR_SHAPE: a step's groups must fit), n_slots <= 32768 and
+ * M <= 8192 (else KVSWAP_ERR_UNSUPPORTED).  KVSWAP_ERR_WORKSPACE if state_bytes is too small.
+ * All calls are asynchronous on `cuda_stream`.
+ */
+size_t kvswap_reuse_state_bytes(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups);
+int kvswap_reuse_init(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, void* state,
+                      size_t state_bytes, void* cuda_stream);
+int kvswap_reuse_lookup(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups,
+                        const int32_t* group_idx, const int32_t* n_selected, void* state,
+                        size_t state_bytes, int32_t* slot_idx, int32_t* miss_group, int32_t* miss_slot,
+                        int32_t* n_miss, void* cuda_stream);
+int kvswap_reuse_fill(const kvswap_shape* shape, int32_t n_slots, const void* K_slow, const void* V_slow,
+                      void* K_reuse, void* V_reuse, const int32_t* miss_group, const int32_t* miss_slot,
+                      const int32_t* n_miss, void* cuda_stream);
+
+/*
  * kvswap_append_kv for every layer of a model at once: k_new, v_new [L, B, H_kv, d] kv_dtype
  * (dense, device) join row N = shape->n_ctx of layers->K[l], layers->V[l] (one launch per 32
  * layers); when that completes a group, each layer's compact-cache rows of the group are built.

@@ -68,6 +68,14 @@ def load() -> ctypes.CDLL:
     lib.kvswap_project_keys.argtypes = [P, V, V, V, I32, I32, V, SZ, V]
     lib.kvswap_append_kv.restype = ctypes.c_int
     lib.kvswap_append_kv.argtypes = [P, V, V, V, V, V, V, ctypes.POINTER(ctypes.c_int32), V]
+    lib.kvswap_reuse_state_bytes.restype = ctypes.c_size_t
+    lib.kvswap_reuse_state_bytes.argtypes = [P, I32, I32]
+    lib.kvswap_reuse_init.restype = ctypes.c_int
+    lib.kvswap_reuse_init.argtypes = [P, I32, I32, V, SZ, V]
+    lib.kvswap_reuse_lookup.restype = ctypes.c_int
+    lib.kvswap_reuse_lookup.argtypes = [P, I32, I32, V, V, V, SZ, V, V, V, V, V]
+    lib.kvswap_reuse_fill.restype = ctypes.c_int
+    lib.kvswap_reuse_fill.argtypes = [P, I32, V, V, V, V, V, V, V, V]
     lib.kvswap_score_select.restype = ctypes.c_int
     lib.kvswap_score_select.argtypes = [P, V, V, V, V, V, V, V, SZ, V]
     lib.kvswap_sparse_decode.restype = ctypes.c_int
@@ -131,6 +139,42 @@ def kvswap_append_kv(shape: kvswap_shape, k_new, v_new, K, V, proj, meta, stream
     _check(load().kvswap_append_kv(ctypes.byref(shape), _ptr(k_new), _ptr(v_new), _ptr(K), _ptr(V), _ptr(proj),
                                    _ptr(meta), ctypes.byref(flushed), _stream(stream)), "kvswap_append_kv")
     return bool(flushed.value)
+
+
+def kvswap_reuse_state_bytes(shape: kvswap_shape, n_slots: int, max_groups: int) -> int:
+    return int(load().kvswap_reuse_state_bytes(ctypes.byref(shape), n_slots, max_groups))
+
+
+def kvswap_reuse_init(shape, n_slots, max_groups, state, stream=None) -> None:
+    _check(load().kvswap_reuse_init(ctypes.byref(shape), n_slots, max_groups, _ptr(state),
+                                    state.numel() * state.element_size(), _stream(stream)), "kvswap_reuse_init")
+
+
+def kvswap_reuse_lookup(shape, n_slots, max_groups, group_idx, n_selected, state, slot_idx, miss_group, miss_slot,
+                        n_miss, stream=None) -> None:
+    _check(load().kvswap_reuse_lookup(ctypes.byref(shape), n_slots, max_groups, _ptr(group_idx), _ptr(n_selected),
+                                      _ptr(state), state.numel() * state.element_size(), _ptr(slot_idx),
+                                      _ptr(miss_group), _ptr(miss_slot), _ptr(n_miss), _stream(stream)),
+           "kvswap_reuse_lookup")
+
+
+def kvswap_reuse_fill(shape, n_slots, K_slow, V_slow, K_reuse, V_reuse, miss_group, miss_slot, n_miss,
+                      stream=None) -> None:
+    """K_slow / V_slow may be CUDA tensors or pinned CPU tensors (read by the GPU in place)."""
+    _check(load().kvswap_reuse_fill(ctypes.byref(shape), n_slots, _ptr(K_slow), _ptr(V_slow), _ptr(K_reuse),
+                                    _ptr(V_reuse), _ptr(miss_group), _ptr(miss_slot), _ptr(n_miss), _stream(stream)),
+           "kvswap_reuse_fill")
+
+
+def reuse_attention_shape(shape: kvswap_shape, n_slots: int) -> kvswap_shape:
+    """The shape that describes the reuse store to kvswap_sparse_decode: n_slots groups plus the
+    rolling-buffer rows, dense [B, H_kv, (n_slots + 1) G, d]."""
+    G, d, Hkv = shape.group_size, shape.head_dim, shape.n_kv_heads
+    R = (n_slots + 1) * G
+    other = kvswap_shape.from_buffer_copy(shape)
+    other.n_ctx = n_slots * G + shape.n_ctx % G
+    other.kv_stride_b, other.kv_stride_h, other.kv_stride_n = Hkv * R * d, R * d, d
+    return other
 
 
 def kvswap_score_select(shape, q, proj, meta, group_idx, n_selected, group_scores_opt, ws, stream=None) -> None:

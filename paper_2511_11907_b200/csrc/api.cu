@@ -227,6 +227,67 @@ int kvswap_append_step(const kvswap_shape* shape, const kvswap_layers* layers, c
   return KVSWAP_OK;
 }
 
+// Checks shared by the reuse-buffer calls.
+static int resolve_reuse(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, Problem* p) {
+  int st = resolve(shape, p);
+  if (st != KVSWAP_OK) return st;
+  if (n_slots < 1 || max_groups < 1 || n_slots < p->M) return KVSWAP_ERR_SHAPE;
+  if (!reuse_supported(*p, n_slots, max_groups)) return KVSWAP_ERR_UNSUPPORTED;
+  return KVSWAP_OK;
+}
+
+size_t kvswap_reuse_state_bytes(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups) {
+  Problem p;
+  if (resolve_reuse(shape, n_slots, max_groups, &p) != KVSWAP_OK) return 0;
+  return sizeof(int32_t) * reuse_state_words(p, n_slots, max_groups);
+}
+
+int kvswap_reuse_init(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, void* state, size_t state_bytes,
+                      void* cuda_stream) {
+  Problem p;
+  int st = resolve_reuse(shape, n_slots, max_groups, &p);
+  if (st != KVSWAP_OK) return st;
+  if (state == nullptr) return KVSWAP_ERR_NULL;
+  if (misaligned(state)) return KVSWAP_ERR_ALIGN;
+  if (state_bytes < sizeof(int32_t) * reuse_state_words(p, n_slots, max_groups)) return KVSWAP_ERR_WORKSPACE;
+  cudaError_t e = launch_reuse_init(p, n_slots, max_groups, static_cast<int32_t*>(state),
+                                    static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+}
+
+int kvswap_reuse_lookup(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, const int32_t* group_idx,
+                        const int32_t* n_selected, void* state, size_t state_bytes, int32_t* slot_idx,
+                        int32_t* miss_group, int32_t* miss_slot, int32_t* n_miss, void* cuda_stream) {
+  Problem p;
+  int st = resolve_reuse(shape, n_slots, max_groups, &p);
+  if (st != KVSWAP_OK) return st;
+  if (group_idx == nullptr || n_selected == nullptr || state == nullptr || slot_idx == nullptr ||
+      miss_group == nullptr || miss_slot == nullptr || n_miss == nullptr)
+    return KVSWAP_ERR_NULL;
+  const void* words[] = {group_idx, n_selected, state, slot_idx, miss_group, miss_slot, n_miss};
+  for (const void* w : words)
+    if (reinterpret_cast<uintptr_t>(w) & 3u) return KVSWAP_ERR_ALIGN;
+  if (state_bytes < sizeof(int32_t) * reuse_state_words(p, n_slots, max_groups)) return KVSWAP_ERR_WORKSPACE;
+  cudaError_t e = launch_reuse_lookup(p, n_slots, max_groups, group_idx, n_selected, static_cast<int32_t*>(state),
+                                      slot_idx, miss_group, miss_slot, n_miss, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+}
+
+int kvswap_reuse_fill(const kvswap_shape* shape, int32_t n_slots, const void* K_slow, const void* V_slow,
+                      void* K_reuse, void* V_reuse, const int32_t* miss_group, const int32_t* miss_slot,
+                      const int32_t* n_miss, void* cuda_stream) {
+  Problem p;
+  int st = resolve_reuse(shape, n_slots, 1, &p);
+  if (st != KVSWAP_OK) return st;
+  if (K_slow == nullptr || V_slow == nullptr || K_reuse == nullptr || V_reuse == nullptr || miss_group == nullptr ||
+      miss_slot == nullptr || n_miss == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (misaligned(K_slow) || misaligned(V_slow) || misaligned(K_reuse) || misaligned(V_reuse)) return KVSWAP_ERR_ALIGN;
+  cudaError_t e = launch_reuse_fill(p, n_slots, K_slow, V_slow, K_reuse, V_reuse, miss_group, miss_slot, n_miss,
+                                    static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+}
+
 int kvswap_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
                         int32_t* group_idx, int32_t* n_selected, float* group_scores_opt, void* ws,
                         size_t ws_bytes, void* cuda_stream) {

@@ -53,6 +53,16 @@ cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* 
                                int n_layers, int n, cudaStream_t st);
 cudaError_t launch_project_keys_layers(const Problem& p, const void* const* K, const float* const* proj,
                                        void* const* meta, int n_layers, int n_begin, int n_end, cudaStream_t st);
+// Reuse buffer (reuse_buffer.cu).
+bool reuse_supported(const Problem& p, int n_slots, int max_groups);
+size_t reuse_state_words(const Problem& p, int n_slots, int max_groups);
+cudaError_t launch_reuse_init(const Problem& p, int n_slots, int max_groups, int32_t* state, cudaStream_t st);
+cudaError_t launch_reuse_lookup(const Problem& p, int n_slots, int max_groups, const int32_t* group_idx,
+                                const int32_t* n_selected, int32_t* state, int32_t* slot_idx, int32_t* miss_group,
+                                int32_t* miss_slot, int32_t* n_miss, cudaStream_t st);
+cudaError_t launch_reuse_fill(const Problem& p, int n_slots, const void* K_slow, const void* V_slow, void* K_reuse,
+                              void* V_reuse, const int32_t* miss_group, const int32_t* miss_slot, const int32_t* n_miss,
+                              cudaStream_t st);
 size_t project_keys_umma_scratch_bytes(const Problem& p);
 bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
                                   int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result);

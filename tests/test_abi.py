@@ -131,6 +131,28 @@ def test_append_kv_validates_before_touching_the_gpu(lib):
     assert lib.kvswap_append_step(ctypes.byref(roomy), ctypes.byref(none), fake, fake, None, None) == 2
 
 
+def test_reuse_buffer_calls_validate_before_touching_the_gpu(lib):
+    s = good_shape()                                       # M = 32, B = 2, S = 2
+    ref = ctypes.byref(s)
+    fake = ctypes.c_void_p(4096)
+    assert kv.kvswap_reuse_state_bytes(s, 64, 256) == 4 * 2 * 2 * (1 + 64 + 256)
+    assert kv.kvswap_reuse_state_bytes(s, 16, 256) == 0                  # fewer slots than a step selects
+    assert kv.kvswap_reuse_state_bytes(s, 64, 0) == 0
+    assert kv.kvswap_reuse_state_bytes(s, 1 << 16, 256) == 0             # beyond the supported slot count
+    assert lib.kvswap_reuse_init(ref, 16, 256, fake, 1 << 20, None) == 2
+    assert lib.kvswap_reuse_init(ref, 1 << 16, 256, fake, 1 << 20, None) == 6
+    assert lib.kvswap_reuse_init(ref, 64, 256, None, 1 << 20, None) == 1
+    assert lib.kvswap_reuse_init(ref, 64, 256, fake, 16, None) == 5
+    assert lib.kvswap_reuse_lookup(ref, 64, 256, None, fake, fake, 1 << 20, fake, fake, fake, fake, None) == 1
+    assert lib.kvswap_reuse_lookup(ref, 64, 256, ctypes.c_void_p(4098), fake, fake, 1 << 20, fake, fake, fake, fake,
+                                   None) == 4
+    assert lib.kvswap_reuse_lookup(ref, 64, 256, fake, fake, fake, 64, fake, fake, fake, fake, None) == 5
+    assert lib.kvswap_reuse_lookup(ref, 8, 256, fake, fake, fake, 1 << 20, fake, fake, fake, fake, None) == 2
+    assert lib.kvswap_reuse_fill(ref, 64, None, fake, fake, fake, fake, fake, fake, None) == 1
+    assert lib.kvswap_reuse_fill(ref, 64, ctypes.c_void_p(4100), fake, fake, fake, fake, fake, fake, None) == 4
+    assert lib.kvswap_reuse_fill(ref, 8, fake, fake, fake, fake, fake, fake, fake, None) == 2
+
+
 def test_status_strings_and_version(lib):
     seen = {kv.status_string(i) for i in range(11)}
     assert len(seen) == 11 and "ok" in seen
