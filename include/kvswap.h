@@ -320,6 +320,42 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
                        void* ws, size_t ws_bytes, const kvswap_probe* probe_opt, void* cuda_stream);
 
 /*
+ * The decode step over a tiered cache (Sec. 4.4.2, Sec. 4.4.3): the full K/V of every layer lives
+ * in a slow tier, each layer has a reuse buffer (kvswap_reuse_* above) in device memory, and the
+ * step's attention reads only reuse stores.  Per layer the internal predictor stream runs
+ * score/select, kvswap_reuse_lookup and kvswap_reuse_fill, so a layer's misses are fetched while
+ * the layers before it are attended on `cuda_stream`; the attention is kvswap_sparse_decode over
+ * the layer's reuse store with the slot list.  Arrays of L per-layer pointers are HOST arrays.
+ *   K_slow, V_slow    [L] slow-tier stores, laid out by shape's kv strides (GPU-readable memory)
+ *   K_reuse, V_reuse  [L] reuse stores [B, H_kv, (n_slots + 1) G, d]; the caller keeps the
+ *                     N mod G newest tokens in rows [n_slots G, n_slots G + N mod G)
+ *   state             [L] reuse-buffer states of state_bytes each (kvswap_reuse_init)
+ *   slot_idx, miss_group, miss_slot [L, B, S, M], n_miss [L, B, S]: device, written by the step
+ * layers->K and layers->V are not used (may be NULL).  `ws` needs
+ * kvswap_tiered_workspace_bytes(shape, n_slots) bytes.  group_idx / n_selected receive the
+ * selections as in kvswap_decode_step.  Errors as for the calls it is made of.
+ */
+typedef struct {
+  int32_t n_slots, max_groups;
+  const void* const* K_slow;
+  const void* const* V_slow;
+  void* const* K_reuse;
+  void* const* V_reuse;
+  void* const* state;
+  size_t state_bytes;
+  int32_t* slot_idx;
+  int32_t* miss_group;
+  int32_t* miss_slot;
+  int32_t* n_miss;
+} kvswap_tiers;
+
+size_t kvswap_tiered_workspace_bytes(const kvswap_shape* shape, int32_t n_slots);
+int kvswap_decode_step_tiered(const kvswap_shape* shape, const kvswap_layers* layers,
+                              const kvswap_tiers* tiers, const void* q, float* out, float* lse_opt,
+                              int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
+                              void* cuda_stream);
+
+/*
  * The same step for callers whose queries and outputs live in HOST memory: q_host
  * [L, B, H_q, d] q_dtype is copied to the device buffer q_dev, the step runs, and out_dev is
  * copied to out_host [L, B, H_q, d] fp32, all asynchronously on `cuda_stream` (use pinned host

@@ -215,6 +215,34 @@ class kvswap_layers(ctypes.Structure):
                 ("proj", ctypes.POINTER(ctypes.c_void_p))]
 
 
+class kvswap_tiers(ctypes.Structure):
+    _fields_ = [("n_slots", ctypes.c_int32), ("max_groups", ctypes.c_int32),
+                ("K_slow", ctypes.POINTER(ctypes.c_void_p)), ("V_slow", ctypes.POINTER(ctypes.c_void_p)),
+                ("K_reuse", ctypes.POINTER(ctypes.c_void_p)), ("V_reuse", ctypes.POINTER(ctypes.c_void_p)),
+                ("state", ctypes.POINTER(ctypes.c_void_p)), ("state_bytes", ctypes.c_size_t),
+                ("slot_idx", ctypes.c_void_p), ("miss_group", ctypes.c_void_p), ("miss_slot", ctypes.c_void_p),
+                ("n_miss", ctypes.c_void_p)]
+
+
+def make_tiers(n_slots, max_groups, K_slow, V_slow, K_reuse, V_reuse, state, slot_idx, miss_group, miss_slot,
+               n_miss) -> kvswap_tiers:
+    """Pointer tables for lists of per-layer tensors (K_slow / V_slow: CUDA or pinned CPU tensors) and the
+    [L, ...] output tensors.  The returned struct keeps everything alive."""
+    n = len(K_slow)
+    assert all(len(x) == n for x in (V_slow, K_reuse, V_reuse, state))
+
+    def table(ts):
+        return (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+
+    tabs = [table(K_slow), table(V_slow), table(K_reuse), table(V_reuse), table(state)]
+    cast = [ctypes.cast(t, ctypes.POINTER(ctypes.c_void_p)) for t in tabs]
+    tiers = kvswap_tiers(int(n_slots), int(max_groups), *cast, state[0].numel() * state[0].element_size(),
+                         slot_idx.data_ptr(), miss_group.data_ptr(), miss_slot.data_ptr(), n_miss.data_ptr())
+    tiers._keep = (tabs, list(K_slow), list(V_slow), list(K_reuse), list(V_reuse), list(state), slot_idx, miss_group,
+                   miss_slot, n_miss)
+    return tiers
+
+
 class kvswap_probe(ctypes.Structure):
     _fields_ = [("layer", ctypes.c_int32), ("ev_begin", ctypes.c_void_p), ("ev_mid", ctypes.c_void_p),
                 ("ev_end", ctypes.c_void_p)]
@@ -257,6 +285,11 @@ def _declare_step(lib):
     lib.kvswap_decode_step.argtypes = [P, PL, V, V, V, V, V, V, SZ, PP, V]
     lib.kvswap_append_step.restype = ctypes.c_int
     lib.kvswap_append_step.argtypes = [P, PL, V, V, ctypes.POINTER(ctypes.c_int32), V]
+    PT = ctypes.POINTER(kvswap_tiers)
+    lib.kvswap_tiered_workspace_bytes.restype = ctypes.c_size_t
+    lib.kvswap_tiered_workspace_bytes.argtypes = [P, ctypes.c_int32]
+    lib.kvswap_decode_step_tiered.restype = ctypes.c_int
+    lib.kvswap_decode_step_tiered.argtypes = [P, PL, PT, V, V, V, V, V, V, SZ, V]
     lib.kvswap_decode_step_host.restype = ctypes.c_int
     lib.kvswap_decode_step_host.argtypes = [P, PL, V, V, V, V, V, V, V, SZ, V]
     lib._step_declared = True
@@ -278,6 +311,17 @@ def kvswap_append_step(shape, layers, k_new, v_new, stream=None) -> bool:
     _check(lib.kvswap_append_step(ctypes.byref(shape), ctypes.byref(layers), _ptr(k_new), _ptr(v_new),
                                   ctypes.byref(flushed), _stream(stream)), "kvswap_append_step")
     return bool(flushed.value)
+
+
+def kvswap_tiered_workspace_bytes(shape, n_slots: int) -> int:
+    return int(_declare_step(load()).kvswap_tiered_workspace_bytes(ctypes.byref(shape), n_slots))
+
+
+def kvswap_decode_step_tiered(shape, layers, tiers, q, out, lse_opt, group_idx, n_selected, ws, stream=None) -> None:
+    lib = _declare_step(load())
+    _check(lib.kvswap_decode_step_tiered(ctypes.byref(shape), ctypes.byref(layers), ctypes.byref(tiers), _ptr(q),
+                                         _ptr(out), _ptr(lse_opt), _ptr(group_idx), _ptr(n_selected), _ptr(ws),
+                                         ws.numel() * ws.element_size(), _stream(stream)), "kvswap_decode_step_tiered")
 
 
 def kvswap_decode_step_host(shape, layers, q_host, out_host, q_dev, out_dev, group_idx, n_selected, ws,

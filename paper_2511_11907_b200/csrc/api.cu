@@ -322,12 +322,23 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
   return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
 }
 
-static int check_layers(const kvswap_layers* layers) {
-  if (layers == nullptr || layers->K == nullptr || layers->V == nullptr || layers->meta == nullptr ||
-      layers->proj == nullptr)
-    return KVSWAP_ERR_NULL;
+static int check_layers(const kvswap_layers* layers, bool need_kv = true) {
+  if (layers == nullptr || layers->meta == nullptr || layers->proj == nullptr) return KVSWAP_ERR_NULL;
+  if (need_kv && (layers->K == nullptr || layers->V == nullptr)) return KVSWAP_ERR_NULL;
   if (layers->n_layers < 1 || layers->max_lookahead < 0) return KVSWAP_ERR_SHAPE;
   return KVSWAP_OK;
+}
+
+// The shape under which kvswap_sparse_decode sees a reuse store: n_slots groups followed by the
+// rolling-buffer rows, dense [B, H_kv, (n_slots + 1) G, d].
+static kvswap_shape reuse_store_shape(const kvswap_shape& s, int32_t n_slots) {
+  kvswap_shape r = s;
+  const int64_t R = int64_t(n_slots + 1) * s.group_size;
+  r.n_ctx = n_slots * s.group_size + s.n_ctx % s.group_size;
+  r.kv_stride_n = s.head_dim;
+  r.kv_stride_h = R * s.head_dim;
+  r.kv_stride_b = int64_t(s.n_kv_heads) * R * s.head_dim;
+  return r;
 }
 
 // Per-device resources of kvswap_decode_step's two-stream schedule: a stream for the predictor and
@@ -376,15 +387,47 @@ cudaError_t step_resources(int n_layers, StepResources** out) {
 }
 }  // namespace
 
-int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q, float* out,
-                       float* lse_opt, int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
-                       const kvswap_probe* probe_opt, void* cuda_stream) {
+// One decode step over all layers; with `tiers` the attention is served from per-layer reuse buffers
+// that the predictor stream keeps filled from the slow tier.
+static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* layers, const kvswap_tiers* tiers,
+                            const void* q, float* out, float* lse_opt, int32_t* group_idx, int32_t* n_selected,
+                            void* ws, size_t ws_bytes, const kvswap_probe* probe_opt, void* cuda_stream) {
   Problem p;
   int st = resolve(shape, &p);
   if (st != KVSWAP_OK) return st;
-  st = check_layers(layers);
+  st = check_layers(layers, tiers == nullptr);
   if (st != KVSWAP_OK) return st;
   if (q == nullptr || out == nullptr || group_idx == nullptr || n_selected == nullptr) return KVSWAP_ERR_NULL;
+  // Tiered: the predictor uses the head of the workspace, the attention over the reuse stores
+  // (another shape, another plan) the part behind it, since the two run on different streams.
+  kvswap_shape shape_attn = *shape;
+  void* ws_attn = ws;
+  size_t ws_attn_bytes = ws_bytes;
+  if (tiers != nullptr) {
+    Problem pr;
+    st = resolve_reuse(shape, tiers->n_slots, tiers->max_groups, &pr);
+    if (st != KVSWAP_OK) return st;
+    if (tiers->K_slow == nullptr || tiers->V_slow == nullptr || tiers->K_reuse == nullptr ||
+        tiers->V_reuse == nullptr || tiers->state == nullptr || tiers->slot_idx == nullptr ||
+        tiers->miss_group == nullptr || tiers->miss_slot == nullptr || tiers->n_miss == nullptr)
+      return KVSWAP_ERR_NULL;
+    if (tiers->state_bytes < sizeof(int32_t) * reuse_state_words(pr, tiers->n_slots, tiers->max_groups))
+      return KVSWAP_ERR_WORKSPACE;
+    for (int l = 0; l < layers->n_layers; ++l) {
+      if (tiers->K_slow[l] == nullptr || tiers->V_slow[l] == nullptr || tiers->K_reuse[l] == nullptr ||
+          tiers->V_reuse[l] == nullptr || tiers->state[l] == nullptr)
+        return KVSWAP_ERR_NULL;
+      if (misaligned(tiers->K_slow[l]) || misaligned(tiers->V_slow[l]) || misaligned(tiers->K_reuse[l]) ||
+          misaligned(tiers->V_reuse[l]) || misaligned(tiers->state[l]))
+        return KVSWAP_ERR_ALIGN;
+    }
+    shape_attn = reuse_store_shape(*shape, tiers->n_slots);
+    const size_t head_bytes = (kvswap_workspace_bytes(shape) + 255) & ~size_t(255);
+    if (ws == nullptr) return KVSWAP_ERR_NULL;
+    if (ws_bytes < head_bytes + kvswap_workspace_bytes(&shape_attn)) return KVSWAP_ERR_WORKSPACE;
+    ws_attn = static_cast<char*>(ws) + head_bytes;
+    ws_attn_bytes = ws_bytes - head_bytes;
+  }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int L = layers->n_layers;
   const size_t q_bytes = size_t(p.B) * p.Hq * p.d * dtype_bytes(p.q_dtype);
@@ -395,8 +438,8 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
                           &p, &w);
   if (st != KVSWAP_OK) return st;
   for (int l = 0; l < L; ++l) {
-    if (layers->proj[l] == nullptr || layers->meta[l] == nullptr || layers->K[l] == nullptr || layers->V[l] == nullptr)
-      return KVSWAP_ERR_NULL;
+    if (layers->proj[l] == nullptr || layers->meta[l] == nullptr) return KVSWAP_ERR_NULL;
+    if (tiers == nullptr && (layers->K[l] == nullptr || layers->V[l] == nullptr)) return KVSWAP_ERR_NULL;
     if (misaligned(layers->proj[l]) || misaligned(layers->meta[l])) return KVSWAP_ERR_ALIGN;
   }
 
@@ -419,7 +462,7 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
   // q is an input of the step (the fork event orders both streams after whatever produced it) and
   // each selection is awaited through its event before the attention that reads it is launched:
   // the inputs of both the predictor and the attention are settled.
-  kvswap_shape shape_settled = *shape;
+  kvswap_shape shape_settled = shape_attn;
   shape_settled.flags |= KVSWAP_INPUTS_SETTLED;
   Problem p_settled = p;
   p_settled.flags |= KVSWAP_INPUTS_SETTLED;
@@ -439,6 +482,20 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
     if (score_select_launch(p_settled, w, ql, layers->proj[l], layers->meta[l], group_idx + size_t(l) * idx_elems,
                             n_selected + size_t(l) * nsel_elems, nullptr, ws, pred) != cudaSuccess)
       return KVSWAP_ERR_CUDA;
+    if (tiers != nullptr) {
+      // Hits keep their slots, misses are fetched from the slow tier -- still on the predictor
+      // stream, so the fetch for this layer overlaps the attention of the layers before it.
+      int32_t* slot_l = tiers->slot_idx + size_t(l) * idx_elems;
+      int32_t* mg_l = tiers->miss_group + size_t(l) * idx_elems;
+      int32_t* ms_l = tiers->miss_slot + size_t(l) * idx_elems;
+      int32_t* nm_l = tiers->n_miss + size_t(l) * nsel_elems;
+      if (launch_reuse_lookup(p, tiers->n_slots, tiers->max_groups, group_idx + size_t(l) * idx_elems,
+                              n_selected + size_t(l) * nsel_elems, static_cast<int32_t*>(tiers->state[l]), slot_l, mg_l,
+                              ms_l, nm_l, pred) != cudaSuccess ||
+          launch_reuse_fill(p, tiers->n_slots, tiers->K_slow[l], tiers->V_slow[l], tiers->K_reuse[l],
+                            tiers->V_reuse[l], mg_l, ms_l, nm_l, pred) != cudaSuccess)
+        return KVSWAP_ERR_CUDA;
+    }
     if (probed && probe_opt->ev_mid) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_mid), pred);
     if (cudaEventRecord(res->selected[l], pred) != cudaSuccess) return KVSWAP_ERR_CUDA;
     return KVSWAP_OK;
@@ -449,9 +506,12 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
       return KVSWAP_ERR_CUDA;
     const bool probed = probe_opt != nullptr && probe_opt->layer == l;
     const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-    const int r = kvswap_sparse_decode(&shape_settled, ql, layers->K[l], layers->V[l], group_idx + size_t(l) * idx_elems,
-                                       n_selected + size_t(l) * nsel_elems, out + size_t(l) * out_elems,
-                                       lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes,
+    const void* Kl = tiers ? tiers->K_reuse[l] : layers->K[l];
+    const void* Vl = tiers ? tiers->V_reuse[l] : layers->V[l];
+    const int32_t* list_l = (tiers ? tiers->slot_idx : group_idx) + size_t(l) * idx_elems;
+    const int r = kvswap_sparse_decode(&shape_settled, ql, Kl, Vl, list_l, n_selected + size_t(l) * nsel_elems,
+                                       out + size_t(l) * out_elems,
+                                       lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws_attn, ws_attn_bytes,
                                        cuda_stream);
     if (probed && probe_opt->ev_end) cudaEventRecord(static_cast<cudaEvent_t>(probe_opt->ev_end), stream);
     if (bounded && r == KVSWAP_OK && cudaEventRecord(res->attended[l], stream) != cudaSuccess)
@@ -476,6 +536,30 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
       return KVSWAP_ERR_CUDA;
   }
   return status;
+}
+
+int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q, float* out,
+                       float* lse_opt, int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
+                       const kvswap_probe* probe_opt, void* cuda_stream) {
+  return decode_step_impl(shape, layers, nullptr, q, out, lse_opt, group_idx, n_selected, ws, ws_bytes, probe_opt,
+                          cuda_stream);
+}
+
+size_t kvswap_tiered_workspace_bytes(const kvswap_shape* shape, int32_t n_slots) {
+  Problem p;
+  if (resolve_reuse(shape, n_slots, 1, &p) != KVSWAP_OK) return 0;
+  const kvswap_shape r = reuse_store_shape(*shape, n_slots);
+  const size_t tail = kvswap_workspace_bytes(&r);
+  if (tail == 0) return 0;
+  return ((kvswap_workspace_bytes(shape) + 255) & ~size_t(255)) + tail;
+}
+
+int kvswap_decode_step_tiered(const kvswap_shape* shape, const kvswap_layers* layers, const kvswap_tiers* tiers,
+                              const void* q, float* out, float* lse_opt, int32_t* group_idx, int32_t* n_selected,
+                              void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (tiers == nullptr) return KVSWAP_ERR_NULL;
+  return decode_step_impl(shape, layers, tiers, q, out, lse_opt, group_idx, n_selected, ws, ws_bytes, nullptr,
+                          cuda_stream);
 }
 
 int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* layers, const void* q_host,

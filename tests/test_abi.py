@@ -153,6 +153,28 @@ def test_reuse_buffer_calls_validate_before_touching_the_gpu(lib):
     assert lib.kvswap_reuse_fill(ref, 8, fake, fake, fake, fake, fake, fake, fake, None) == 2
 
 
+def test_tiered_step_validates_before_touching_the_gpu(lib):
+    kv._declare_step(lib)
+    s = good_shape()
+    assert kv.kvswap_tiered_workspace_bytes(s, 64) > kv.kvswap_workspace_bytes(s)
+    assert kv.kvswap_tiered_workspace_bytes(s, 8) == 0
+    fake = ctypes.c_void_p(4096)
+    tab = (ctypes.c_void_p * 1)(4096)
+    ptab = ctypes.cast(tab, ctypes.POINTER(ctypes.c_void_p))
+    layers = kv.kvswap_layers(1, 0, None, None, ptab, ptab)               # K and V tables are not needed
+    tiers = kv.kvswap_tiers(64, 256, ptab, ptab, ptab, ptab, ptab, 1 << 20, 4096, 4096, 4096, 4096)
+    call = lambda t, ws_bytes: lib.kvswap_decode_step_tiered(ctypes.byref(s), ctypes.byref(layers), t, fake, fake, None,
+                                                             fake, fake, fake, ws_bytes, None)
+    assert call(None, 1 << 30) == 1
+    assert call(ctypes.byref(tiers), 1024) == 5                            # workspace too small
+    small_state = kv.kvswap_tiers(64, 256, ptab, ptab, ptab, ptab, ptab, 64, 4096, 4096, 4096, 4096)
+    assert call(ctypes.byref(small_state), 1 << 30) == 5
+    few_slots = kv.kvswap_tiers(8, 256, ptab, ptab, ptab, ptab, ptab, 1 << 20, 4096, 4096, 4096, 4096)
+    assert call(ctypes.byref(few_slots), 1 << 30) == 2
+    no_out = kv.kvswap_tiers(64, 256, ptab, ptab, ptab, ptab, ptab, 1 << 20, None, 4096, 4096, 4096)
+    assert call(ctypes.byref(no_out), 1 << 30) == 1
+
+
 def test_status_strings_and_version(lib):
     seen = {kv.status_string(i) for i in range(11)}
     assert len(seen) == 11 and "ok" in seen

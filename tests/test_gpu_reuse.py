@@ -183,3 +183,66 @@ def test_attention_from_the_reuse_buffer_all_heads_scope_fp32():
 def test_attention_from_the_reuse_buffer_group_of_sixteen():
     wl = W.REDUCED[4].reduced("cfg4-reuse", n_ctx=4096 + 9)
     _tiered_attention_case(wl, 1, KV, n_slots=40, steps=3)
+
+
+@pytest.mark.parametrize("lookahead", [0, 1])
+def test_tiered_decode_step_matches_the_step_over_the_full_store(lookahead):
+    """Four layers, slow tier in pinned host memory, three consecutive steps (the reuse buffers carry
+    over): outputs agree with kvswap_decode_step over the HBM-resident stores, selections are
+    identical, every slot list points at slots holding the selected groups."""
+    from paper_2511_11907_b200 import device_workload as DW
+    wl = W.REDUCED[5].reduced("cfg5-tiered", layers=4, n_ctx=4096 + 3, top_k=48, walk_steps=3)
+    dw = DW.build(wl, 1, KV, walk_steps=3, reserve_bytes=1 << 30)
+    shape, L = dw.shape, wl.layers
+    B, Hkv, N, d, G, M = wl.batch, wl.n_kv_heads, wl.n_ctx, wl.head_dim, wl.group_size, wl.top_k
+    NG, S, C = N // G, shape.n_scopes, 80
+    ws = rt.alloc_workspace(shape)
+    for l in range(L):
+        kv.kvswap_project_keys(shape, dw.K[l], dw.proj[l], dw.meta[l], 0, N, ws)
+    K_slow = [k.cpu().pin_memory() for k in dw.K]
+    V_slow = [v.cpu().pin_memory() for v in dw.V]
+    R = (C + 1) * G
+    K_r = [torch.full((B, Hkv, R, d), float("nan"), dtype=dw.K[0].dtype, device="cuda") for _ in range(L)]
+    V_r = [torch.full((B, Hkv, R, d), float("nan"), dtype=dw.K[0].dtype, device="cuda") for _ in range(L)]
+    for l in range(L):
+        K_r[l][:, :, C * G:C * G + N % G] = dw.K[l][:, :, NG * G:]
+        V_r[l][:, :, C * G:C * G + N % G] = dw.V[l][:, :, NG * G:]
+    n_state = kv.kvswap_reuse_state_bytes(shape, C, NG) // 4
+    state = [torch.empty(n_state, dtype=torch.int32, device="cuda") for _ in range(L)]
+    for l in range(L):
+        kv.kvswap_reuse_init(shape, C, NG, state[l])
+    slot_idx = torch.full((L, B, S, M), -9, dtype=torch.int32, device="cuda")
+    miss_group, miss_slot = torch.full_like(slot_idx, -9), torch.full_like(slot_idx, -9)
+    n_miss = torch.full((L, B, S), -9, dtype=torch.int32, device="cuda")
+    tiers = kv.make_tiers(C, NG, K_slow, V_slow, K_r, V_r, state, slot_idx, miss_group, miss_slot, n_miss)
+    layers_hbm = dw.layer_tables(lookahead)
+    layers_tiered = kv.make_layers(K_r, V_r, dw.meta, dw.proj, lookahead)
+    ws_t = torch.empty(kv.kvswap_tiered_workspace_bytes(shape, C), dtype=torch.uint8, device="cuda")
+    kv.kvswap_workspace_init(ws_t)
+    mk = lambda: (torch.full((L, B, wl.n_q_heads, d), float("nan"), device="cuda"),
+                  torch.full((L, B, wl.n_q_heads), float("nan"), device="cuda"),
+                  torch.full((L, B, S, M), -7, dtype=torch.int32, device="cuda"),
+                  torch.full((L, B, S), -7, dtype=torch.int32, device="cuda"))
+    missed = []
+    for t in range(3):
+        q = dw.q_walk[t]
+        out_a, lse_a, idx_a, nsel_a = mk()
+        kv.kvswap_decode_step(shape, layers_hbm, q, out_a, lse_a, idx_a, nsel_a, ws)
+        out_b, lse_b, idx_b, nsel_b = mk()
+        kv.kvswap_decode_step_tiered(shape, layers_tiered, tiers, q, out_b, lse_b, idx_b, nsel_b, ws_t)
+        torch.cuda.synchronize()
+        assert kv.kvswap_read_device_status(ws_t) == 0
+        assert torch.equal(idx_a, idx_b) and torch.equal(nsel_a, nsel_b)
+        tol = OUT_ATOL_TIGHT[wl.kv_dtype]
+        assert (out_a - out_b).abs().max().item() <= tol and (lse_a - lse_b).abs().max().item() <= tol
+        sl, ix = slot_idx.cpu().numpy(), idx_b.cpu().numpy()
+        assert sl.min() >= 0 and sl.max() < C
+        for l in range(L):
+            for b in range(B):
+                for s in range(S):
+                    assert len(set(sl[l, b, s].tolist())) == M                   # no slot serves two groups
+                    for i in (0, M - 1):
+                        j, c = int(ix[l, b, s, i]), int(sl[l, b, s, i])
+                        assert torch.equal(K_r[l][b, s, c * G:(c + 1) * G], dw.K[l][b, s, j * G:(j + 1) * G])
+        missed.append(int(n_miss.sum().item()))
+    assert missed[0] == L * B * S * M and missed[1] < missed[0] and missed[2] < missed[0]
