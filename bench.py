@@ -454,6 +454,38 @@ def run_ours(args, wl):
                      "fill_gbs_from_host": statistics.mean(fill_bytes[warm]) / statistics.mean(t_fill[warm]) / 1e6,
                      "attention_from_slots_us": 1e3 * statistics.mean(t_att[warm])}
             del K_slow, V_slow, K_r, V_r
+            # the same through kvswap_decode_step_tiered over the first layers of the model: lookup and miss
+            # gather run on the predictor stream, ahead of the attention of the layers before
+            Lt = min(L, 4)
+            pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+            Ks, Vs = [pin(dw.K[l]) for l in range(Lt)], [pin(dw.V[l]) for l in range(Lt)]
+            Kr = [torch.zeros((wl.batch, Hkv, Rr, d_), dtype=kv_t, device=dev) for _ in range(Lt)]
+            Vr = [torch.zeros((wl.batch, Hkv, Rr, d_), dtype=kv_t, device=dev) for _ in range(Lt)]
+            for l in range(Lt):
+                Kr[l][:, :, C_ * G_:C_ * G_ + tail_] = dw.K[l][:, :, NG_ * G_:]
+                Vr[l][:, :, C_ * G_:C_ * G_ + tail_] = dw.V[l][:, :, NG_ * G_:]
+            states = [torch.empty_like(state) for _ in range(Lt)]
+            for st_l in states:
+                kv.kvswap_reuse_init(shape, C_, NG_, st_l)
+            sl_t = torch.empty((Lt, wl.batch, S, M_), dtype=torch.int32, device=dev)
+            mg_t, ms_t = torch.empty_like(sl_t), torch.empty_like(sl_t)
+            nm_t = torch.empty((Lt, wl.batch, S), dtype=torch.int32, device=dev)
+            tiers = kv.make_tiers(C_, NG_, Ks, Vs, Kr, Vr, states, sl_t, mg_t, ms_t, nm_t)
+            layers_t = kv.make_layers(Kr, Vr, dw.meta[:Lt], dw.proj[:Lt])
+            ws_t = torch.empty(kv.kvswap_tiered_workspace_bytes(shape, C_), dtype=torch.uint8, device=dev)
+            kv.kvswap_workspace_init(ws_t)
+            step_ms, step_rate = [], []
+            for t in range(min(n_walk, 16)):
+                ev[0].record()
+                kv.kvswap_decode_step_tiered(shape, layers_t, tiers, dw.q_walk[t][:Lt], out[:Lt], None, idx[:Lt],
+                                             nsel[:Lt], ws_t)
+                ev[1].record()
+                torch.cuda.synchronize()
+                step_ms.append(ev[0].elapsed_time(ev[1]))
+                step_rate.append(1.0 - int(nm_t.sum().item()) / (Lt * wl.batch * S * min(M_, NG_)))
+            reuse["tiered_step"] = {"layers": Lt, "steps": len(step_ms), "ms_per_layer": statistics.mean(step_ms[warm]) / Lt,
+                                    "ms_per_layer_cold": step_ms[0] / Lt, "reuse_rate_mean": statistics.mean(step_rate[warm])}
+            del Ks, Vs, Kr, Vr
 
     # ---- max over ranks ----------------------------------------------------------------------------
     elapsed_ms, e2e_ms, look1_ms, grow_ms, append_ms = shard.max_over_ranks(
