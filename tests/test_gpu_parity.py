@@ -184,6 +184,11 @@ EDGE = {
                             n_q_heads=6, n_kv_heads=2, n_ctx=8 * 90 + 3, top_k=12),
     "bf16_rank_64": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=64, group_size=8,
                           n_ctx=8 * 64 + 1, top_k=10),
+    "bf16_rank_16": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=16, group_size=8,
+                          n_ctx=8 * 64 + 1, top_k=10),
+    "bf16_rank_128": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=128, group_size=8,
+                           n_ctx=8 * 64 + 1, top_k=10),
+    "rank_128_fp32": small(rank=128, head_dim=128),
     "bf16_gqa_ratio_8": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, group_size=8,
                               n_q_heads=16, n_kv_heads=2, n_ctx=8 * 70 + 5, top_k=14),
     "bf16_gqa_ratio_5": small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=64, rank=32, group_size=4,
