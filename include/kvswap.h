@@ -356,6 +356,19 @@ int kvswap_decode_step_tiered(const kvswap_shape* shape, const kvswap_layers* la
                               void* cuda_stream);
 
 /*
+ * kvswap_append_step for the tiered cache (Sec. 4.4.1 over Sec. 4.4.2).  shape->n_ctx is N before
+ * the call and shape's kv strides describe the slow-tier stores, which need room for row N (as
+ * in kvswap_append_kv).  k_new, v_new [L, B, H_kv, d] join the rolling-buffer rows of each
+ * layer's reuse store (row n_slots G + N mod G).  When the token completes a group, the group's
+ * G rows are written from there to rows [N+1-G, N] of the slow tier (this call WRITES K_slow and
+ * V_slow) and its compact-cache rows are built.  Of `tiers` only n_slots, K_slow, V_slow,
+ * K_reuse and V_reuse are used.  Asynchronous on `cuda_stream`.
+ */
+int kvswap_append_step_tiered(const kvswap_shape* shape, const kvswap_layers* layers,
+                              const kvswap_tiers* tiers, const void* k_new, const void* v_new,
+                              int32_t* flushed_opt, void* cuda_stream);
+
+/*
  * The same step for callers whose queries and outputs live in HOST memory: q_host
  * [L, B, H_q, d] q_dtype is copied to the device buffer q_dev, the step runs, and out_dev is
  * copied to out_host [L, B, H_q, d] fp32, all asynchronously on `cuda_stream` (use pinned host

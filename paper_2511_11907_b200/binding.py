@@ -290,6 +290,8 @@ def _declare_step(lib):
     lib.kvswap_tiered_workspace_bytes.argtypes = [P, ctypes.c_int32]
     lib.kvswap_decode_step_tiered.restype = ctypes.c_int
     lib.kvswap_decode_step_tiered.argtypes = [P, PL, PT, V, V, V, V, V, V, SZ, V]
+    lib.kvswap_append_step_tiered.restype = ctypes.c_int
+    lib.kvswap_append_step_tiered.argtypes = [P, PL, PT, V, V, ctypes.POINTER(ctypes.c_int32), V]
     lib.kvswap_decode_step_host.restype = ctypes.c_int
     lib.kvswap_decode_step_host.argtypes = [P, PL, V, V, V, V, V, V, V, SZ, V]
     lib._step_declared = True
@@ -322,6 +324,15 @@ def kvswap_decode_step_tiered(shape, layers, tiers, q, out, lse_opt, group_idx, 
     _check(lib.kvswap_decode_step_tiered(ctypes.byref(shape), ctypes.byref(layers), ctypes.byref(tiers), _ptr(q),
                                          _ptr(out), _ptr(lse_opt), _ptr(group_idx), _ptr(n_selected), _ptr(ws),
                                          ws.numel() * ws.element_size(), _stream(stream)), "kvswap_decode_step_tiered")
+
+
+def kvswap_append_step_tiered(shape, layers, tiers, k_new, v_new, stream=None) -> bool:
+    lib = _declare_step(load())
+    flushed = ctypes.c_int32(0)
+    _check(lib.kvswap_append_step_tiered(ctypes.byref(shape), ctypes.byref(layers), ctypes.byref(tiers), _ptr(k_new),
+                                         _ptr(v_new), ctypes.byref(flushed), _stream(stream)),
+           "kvswap_append_step_tiered")
+    return bool(flushed.value)
 
 
 def kvswap_decode_step_host(shape, layers, q_host, out_host, q_dev, out_dev, group_idx, n_selected, ws,

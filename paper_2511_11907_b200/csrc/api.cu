@@ -562,6 +562,53 @@ int kvswap_decode_step_tiered(const kvswap_shape* shape, const kvswap_layers* la
                           cuda_stream);
 }
 
+int kvswap_append_step_tiered(const kvswap_shape* shape, const kvswap_layers* layers, const kvswap_tiers* tiers,
+                              const void* k_new, const void* v_new, int32_t* flushed_opt, void* cuda_stream) {
+  if (flushed_opt != nullptr) *flushed_opt = 0;
+  Problem p;                                   // the grown context: N + 1 tokens, the slow tier's strides
+  int st = resolve_grown(shape, &p);
+  if (st != KVSWAP_OK) return st;
+  st = check_layers(layers, false);
+  if (st != KVSWAP_OK) return st;
+  if (tiers == nullptr || tiers->K_slow == nullptr || tiers->V_slow == nullptr || tiers->K_reuse == nullptr ||
+      tiers->V_reuse == nullptr || k_new == nullptr || v_new == nullptr)
+    return KVSWAP_ERR_NULL;
+  if (tiers->n_slots < 1) return KVSWAP_ERR_SHAPE;
+  if (misaligned(k_new) || misaligned(v_new)) return KVSWAP_ERR_ALIGN;
+  const int L = layers->n_layers;
+  for (int l = 0; l < L; ++l) {
+    if (tiers->K_slow[l] == nullptr || tiers->V_slow[l] == nullptr || tiers->K_reuse[l] == nullptr ||
+        tiers->V_reuse[l] == nullptr || layers->meta[l] == nullptr || layers->proj[l] == nullptr)
+      return KVSWAP_ERR_NULL;
+    if (misaligned(tiers->K_slow[l]) || misaligned(tiers->V_slow[l]) || misaligned(tiers->K_reuse[l]) ||
+        misaligned(tiers->V_reuse[l]) || misaligned(layers->meta[l]) || misaligned(layers->proj[l]))
+      return KVSWAP_ERR_ALIGN;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // The new token joins the rolling-buffer rows of every layer's reuse store.
+  const int64_t fast_rows = int64_t(tiers->n_slots + 1) * p.G;
+  const int n = p.N - 1;                       // its position in the context
+  Problem fast = p;
+  fast.kv_sn = p.d;
+  fast.kv_sh = fast_rows * p.d;
+  fast.kv_sb = int64_t(p.Hkv) * fast.kv_sh;
+  if (launch_append_rows(fast, k_new, v_new, tiers->K_reuse, tiers->V_reuse, L, tiers->n_slots * p.G + n % p.G,
+                         stream) != cudaSuccess)
+    return KVSWAP_ERR_CUDA;
+  if (p.N % p.G == 0) {
+    // The group is complete: its rows go to the slow tier, and its compact-cache rows are built
+    // from there (the projection reads the rows it was just handed; same stream).
+    if (launch_flush_rows(p, tiers->K_reuse, tiers->V_reuse, const_cast<void* const*>(tiers->K_slow),
+                          const_cast<void* const*>(tiers->V_slow), L, fast_rows, int64_t(tiers->n_slots) * p.G,
+                          p.N - p.G, stream) != cudaSuccess ||
+        launch_project_keys_layers(p, tiers->K_slow, layers->proj, const_cast<void* const*>(layers->meta), L,
+                                   p.N - p.G, p.N, stream) != cudaSuccess)
+      return KVSWAP_ERR_CUDA;
+    if (flushed_opt != nullptr) *flushed_opt = 1;
+  }
+  return KVSWAP_OK;
+}
+
 int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* layers, const void* q_host,
                             float* out_host, void* q_dev, float* out_dev, int32_t* group_idx,
                             int32_t* n_selected, void* ws, size_t ws_bytes, void* cuda_stream) {

@@ -53,6 +53,9 @@ cudaError_t launch_append_rows(const Problem& p, const void* k_new, const void* 
                                int n_layers, int n, cudaStream_t st);
 cudaError_t launch_project_keys_layers(const Problem& p, const void* const* K, const float* const* proj,
                                        void* const* meta, int n_layers, int n_begin, int n_end, cudaStream_t st);
+cudaError_t launch_flush_rows(const Problem& p, const void* const* K_fast, const void* const* V_fast, void* const* K_slow,
+                              void* const* V_slow, int n_layers, int64_t fast_rows, int64_t fast_row0, int64_t slow_row0,
+                              cudaStream_t st);
 // Reuse buffer (reuse_buffer.cu).
 bool reuse_supported(const Problem& p, int n_slots, int max_groups);
 size_t reuse_state_words(const Problem& p, int n_slots, int max_groups);

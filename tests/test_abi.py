@@ -173,6 +173,14 @@ def test_tiered_step_validates_before_touching_the_gpu(lib):
     assert call(ctypes.byref(few_slots), 1 << 30) == 2
     no_out = kv.kvswap_tiers(64, 256, ptab, ptab, ptab, ptab, ptab, 1 << 20, None, 4096, 4096, 4096)
     assert call(ctypes.byref(no_out), 1 << 30) == 1
+    # tiered append: capacity rule as for kvswap_append_kv, then the tables
+    N, d, r = 1024, 64, 16
+    roomy = good_shape(kv_strides=(2 * (N + 8) * d, (N + 8) * d, d), meta_strides=((N + 8) * r, (N + 8) * r, r))
+    app = lambda sh, t: lib.kvswap_append_step_tiered(ctypes.byref(sh), ctypes.byref(layers), t, fake, fake, None, None)
+    assert app(s, ctypes.byref(tiers)) == 2                                # dense strides: no room stated
+    assert app(roomy, None) == 1
+    no_store = kv.kvswap_tiers(64, 256, ptab, ptab, None, ptab, ptab, 1 << 20, 4096, 4096, 4096, 4096)
+    assert app(roomy, ctypes.byref(no_store)) == 1
 
 
 def test_status_strings_and_version(lib):

@@ -246,3 +246,80 @@ def test_tiered_decode_step_matches_the_step_over_the_full_store(lookahead):
                         assert torch.equal(K_r[l][b, s, c * G:(c + 1) * G], dw.K[l][b, s, j * G:(j + 1) * G])
         missed.append(int(n_miss.sum().item()))
     assert missed[0] == L * B * S * M and missed[1] < missed[0] and missed[2] < missed[0]
+
+
+def test_tiered_growing_context_matches_the_hbm_resident_one():
+    """Three layers; the context grows over two group boundaries.  Side A keeps everything in HBM
+    (kvswap_append_step + kvswap_decode_step); side B keeps the full cache in pinned host memory
+    (kvswap_append_step_tiered + kvswap_decode_step_tiered).  Same selections, same attention, and
+    the slow tier ends up holding the appended rows of every completed group."""
+    from paper_2511_11907_b200 import device_workload as DW
+    cap = 2048 + 24
+    wl = W.REDUCED[5].reduced("cfg5-tiered-grow", layers=3, n_ctx=cap, top_k=40, walk_steps=2)
+    dw = DW.build(wl, 1, KV, walk_steps=2, reserve_bytes=1 << 30)
+    L, B, Hkv, d, r, G, M = wl.layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.rank, wl.group_size, wl.top_k
+    n0, steps, C = 2048 + 3, 19, 64
+    strides = dict(kv_strides=(Hkv * cap * d, cap * d, d), meta_strides=(cap * r, cap * r, r))
+    shape_at = lambda n: rt.shape_for(wl, 1, KV, n_ctx=n, **strides)
+    S, NGcap = shape_at(cap).n_scopes, cap // G
+    ws = rt.alloc_workspace(shape_at(cap))
+    gen = torch.Generator(device="cuda").manual_seed(9)
+    new_k = torch.randn((steps, L, B, Hkv, d), generator=gen, device="cuda").to(torch.bfloat16)
+    new_v = torch.randn((steps, L, B, Hkv, d), generator=gen, device="cuda").to(torch.bfloat16)
+    # side A: HBM stores (rows >= n0 poisoned), side B: slow tier in host memory + reuse stores
+    for l in range(L):
+        dw.K[l][:, :, n0:] = float("nan")
+        dw.V[l][:, :, n0:] = float("nan")
+    meta_a = [torch.full((B, 1, cap, r), float("nan"), dtype=torch.float16, device="cuda") for _ in range(L)]
+    meta_b = [m.clone() for m in meta_a]
+    for l in range(L):
+        kv.kvswap_project_keys(shape_at(n0), dw.K[l], dw.proj[l], meta_a[l], 0, n0 // G * G, ws)
+        meta_b[l].copy_(meta_a[l])
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+    K_slow, V_slow = [pin(k) for k in dw.K], [pin(v) for v in dw.V]
+    R = (C + 1) * G
+    K_r = [torch.full((B, Hkv, R, d), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    V_r = [torch.full((B, Hkv, R, d), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    for l in range(L):                                                   # the open group starts in the rolling rows
+        K_r[l][:, :, C * G:C * G + n0 % G] = dw.K[l][:, :, n0 // G * G:n0]
+        V_r[l][:, :, C * G:C * G + n0 % G] = dw.V[l][:, :, n0 // G * G:n0]
+    state = [torch.empty(kv.kvswap_reuse_state_bytes(shape_at(cap), C, NGcap) // 4, dtype=torch.int32, device="cuda")
+             for _ in range(L)]
+    for l in range(L):
+        kv.kvswap_reuse_init(shape_at(cap), C, NGcap, state[l])
+    slot_idx = torch.empty((L, B, S, M), dtype=torch.int32, device="cuda")
+    mg, ms = torch.empty_like(slot_idx), torch.empty_like(slot_idx)
+    nm = torch.empty((L, B, S), dtype=torch.int32, device="cuda")
+    tiers = kv.make_tiers(C, NGcap, K_slow, V_slow, K_r, V_r, state, slot_idx, mg, ms, nm)
+    layers_a = kv.make_layers(dw.K, dw.V, meta_a, dw.proj)
+    layers_b = kv.make_layers(K_r, V_r, meta_b, dw.proj)
+    ws_t = torch.empty(kv.kvswap_tiered_workspace_bytes(shape_at(cap), C), dtype=torch.uint8, device="cuda")
+    kv.kvswap_workspace_init(ws_t)
+    mk = lambda: (torch.full((L, B, wl.n_q_heads, d), float("nan"), device="cuda"),
+                  torch.full((L, B, S, M), -7, dtype=torch.int32, device="cuda"),
+                  torch.full((L, B, S), -7, dtype=torch.int32, device="cuda"))
+    flushes = 0
+    for t in range(steps):
+        n = n0 + t
+        fa = kv.kvswap_append_step(shape_at(n), layers_a, new_k[t], new_v[t])
+        fb = kv.kvswap_append_step_tiered(shape_at(n), layers_b, tiers, new_k[t], new_v[t])
+        assert fa == fb == ((n + 1) % G == 0)
+        flushes += fb
+        q = dw.q_walk[t % 2]
+        out_a, idx_a, nsel_a = mk()
+        out_b, idx_b, nsel_b = mk()
+        kv.kvswap_decode_step(shape_at(n + 1), layers_a, q, out_a, None, idx_a, nsel_a, ws)
+        kv.kvswap_decode_step_tiered(shape_at(n + 1), layers_b, tiers, q, out_b, None, idx_b, nsel_b, ws_t)
+        torch.cuda.synchronize()
+        assert torch.equal(idx_a, idx_b) and torch.equal(nsel_a, nsel_b)
+        assert not torch.isnan(out_b).any()
+        assert (out_a - out_b).abs().max().item() <= OUT_ATOL_TIGHT[wl.kv_dtype]
+    assert flushes == 2
+    n_end = n0 + steps
+    done = n_end // G * G                                                # rows of complete groups
+    for l in range(L):
+        assert torch.equal(K_slow[l][:, :, :done], dw.K[l][:, :, :done].cpu())
+        assert torch.equal(V_slow[l][:, :, :done], dw.V[l][:, :, :done].cpu())
+        assert torch.isnan(K_slow[l][:, :, done:].float()).all()         # the open group is not in the slow tier
+        assert torch.equal(meta_a[l][:, :, :done].view(torch.int16), meta_b[l][:, :, :done].view(torch.int16))
+        assert torch.equal(K_r[l][:, :, C * G:C * G + n_end % G], dw.K[l][:, :, done:n_end])
