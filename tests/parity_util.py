@@ -39,7 +39,7 @@ def project_tolerance(K, proj, meta_heads, oracle_meta, meta_dtype):
 
 
 def check_selection(R, idx_gpu, nsel_gpu, M):
-    """North-star comparator: bit-exact group selection except inside the tie band.
+    """The selection comparator: bit-exact group selection except inside the tie band.
     R: oracle group scores [B,S,NG]; idx_gpu [B,S,M]; nsel_gpu [B,S].  Returns #problems that had
     more than one group inside the band."""
     B, S, NG = R.shape
