@@ -312,9 +312,60 @@ bool try_launch_mma(const Problem& p, const void* K, const float* proj, void* me
   return true;
 }
 
+// A handful of tokens (one flushed group, for every layer): one CTA per (token, sequence, metadata
+// head, layer).  Eight slices of the contraction index x 32 output columns; every thread keeps up
+// to eight columns (r <= 256); the slices are summed through shared memory in a fixed order.
+constexpr int kGroupTokens = 64;              // token ranges up to this length take this kernel
+
+template <typename KV_T, typename META_T>
+__global__ void __launch_bounds__(256)
+project_group_kernel(Problem p, const ProjectTable tab, int n_begin, int n_tokens) {
+  __shared__ float part_sum[8][256];
+  const int layer = blockIdx.x / n_tokens, n = n_begin + blockIdx.x % n_tokens;
+  const int b = blockIdx.y, head_out = blockIdx.z;
+  const KV_T* __restrict__ K = static_cast<const KV_T*>(tab.K[layer]);
+  const float* __restrict__ proj = tab.proj[layer];
+  META_T* __restrict__ meta = static_cast<META_T*>(tab.meta[layer]);
+  const int g_first = (p.Hm == 1) ? 0 : head_out;
+  const int g_count = (p.Hm == 1) ? p.Hkv : 1;
+  const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  const int per_part = p.d / 8;                                  // d is 64 or 128
+  for (int gi = 0; gi < g_count; ++gi) {
+    const int g = g_first + gi;
+    const KV_T* row = K + int64_t(b) * p.kv_sb + int64_t(g) * p.kv_sh + int64_t(n) * p.kv_sn;
+    const float* Pg = proj + int64_t(g) * p.d * p.r;
+    for (int c = part * per_part; c < (part + 1) * per_part; ++c) {
+      const float k = float(row[c]);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int col = lane + 32 * j;
+        if (col < p.r) acc[j] = fmaf(k, Pg[int64_t(c) * p.r + col], acc[j]);
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) part_sum[part][lane + 32 * j] = acc[j];
+  __syncthreads();
+  for (int col = threadIdx.x; col < p.r; col += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += part_sum[k][col];
+    META_T* out = meta + int64_t(b) * p.meta_sb + int64_t(head_out) * p.meta_sh + int64_t(n) * p.meta_sn + col;
+    if constexpr (sizeof(META_T) == 2) *out = __float2half_rn(s); else *out = s;
+  }
+}
+
 template <typename KV_T, typename META_T>
 cudaError_t dispatch_rc(const Problem& p, const ProjectTable& tab, int n_layers, int n_begin, int n_end,
                         cudaStream_t st) {
+  if (n_end - n_begin <= kGroupTokens) {
+    const int n_tokens = n_end - n_begin;
+    project_group_kernel<KV_T, META_T><<<dim3(n_tokens * n_layers, p.B, p.Hm), 256, 0, st>>>(p, tab, n_begin, n_tokens);
+    return cudaGetLastError();
+  }
   const int tiles = (n_end - n_begin + kTok - 1) / kTok;
   dim3 grid(tiles * n_layers, p.B, p.Hm);
   const int rc = (p.r + 31) / 32;
