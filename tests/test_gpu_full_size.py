@@ -76,3 +76,37 @@ def test_full_size_layer_sampled_sequence(cfg, meta_heads):
     assert eo <= OUT_ATOL_TIGHT[wl.kv_dtype] and el <= OUT_ATOL_TIGHT[wl.kv_dtype], (eo, el)
     assert np.all(np.isfinite(out.cpu().numpy()))                 # every other sequence ran too
     assert kv.kvswap_read_device_status(ws) == 0
+
+
+@pytest.mark.parametrize("cfg,lookahead", [(5, 0), (5, 1), (4, 0)])
+def test_full_size_decode_step_equals_the_per_layer_calls(cfg, lookahead):
+    """The call the benchmark times, at its shapes (six layers of the configuration): predictor and
+    attention on two streams, settled launches, waits joined per two layers -- and exactly the
+    results of the per-layer calls, which the test above ties to the oracle."""
+    L = 6
+    wl = W.CONFIGS[cfg].reduced(f"cfg{cfg}-six-layers", layers=L, walk_steps=2)
+    dw = DW.build(wl, 1, W.SCOPE_KV_HEAD)
+    assert dw.layers_resident == L
+    shape = dw.shape
+    ws = rt.alloc_workspace(shape)
+    for l in range(L):
+        kv.kvswap_project_keys(shape, dw.K[l], dw.proj[l], dw.meta[l], 0, wl.n_ctx, ws)
+    B, S, M = wl.batch, shape.n_scopes, wl.top_k
+    mk = lambda: (torch.full((L, B, wl.n_q_heads, wl.head_dim), float("nan"), device="cuda"),
+                  torch.full((L, B, wl.n_q_heads), float("nan"), device="cuda"),
+                  torch.full((L, B, S, M), -7, dtype=torch.int32, device="cuda"),
+                  torch.full((L, B, S), -7, dtype=torch.int32, device="cuda"))
+    layers = dw.layer_tables(lookahead)
+    for step in range(2):
+        q = dw.q_walk[step]
+        out_a, lse_a, idx_a, nsel_a = mk()
+        for l in range(L):
+            kv.kvswap_score_select(shape, q[l], dw.proj[l], dw.meta[l], idx_a[l], nsel_a[l], None, ws)
+            kv.kvswap_sparse_decode(shape, q[l], dw.K[l], dw.V[l], idx_a[l], nsel_a[l], out_a[l], lse_a[l], ws)
+        out_b, lse_b, idx_b, nsel_b = mk()
+        kv.kvswap_decode_step(shape, layers, q, out_b, lse_b, idx_b, nsel_b, ws)
+        kv.kvswap_decode_step(shape, layers, q, out_b, lse_b, idx_b, nsel_b, ws)      # back to back, as in the bench
+        torch.cuda.synchronize()
+        assert kv.kvswap_read_device_status(ws) == 0
+        assert torch.equal(idx_a, idx_b) and torch.equal(nsel_a, nsel_b)
+        assert torch.equal(out_a, out_b) and torch.equal(lse_a, lse_b)
