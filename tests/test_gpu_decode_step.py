@@ -101,3 +101,38 @@ def test_decode_step_fp32_wide_rank_per_head():
     wl = W.CONFIGS[1].reduced("cfg1-wide", layers=6, batch=64, n_ctx=512, rank=128, head_dim=128, n_q_heads=32,
                               n_kv_heads=8, top_k=8, calib_rows=1536)
     _run_case(wl, "per_head", W.SCOPE_KV_HEAD)
+
+
+def test_decode_step_can_be_captured_in_a_cuda_graph():
+    """After a warm-up call (which creates the internal stream and events) the step records into a
+    CUDA graph -- the internal stream forks from and joins the capturing stream -- and replays give
+    the results of the stream-ordered call."""
+    wl = W.CONFIGS[3].reduced("cfg3-graph", layers=4, batch=2, n_ctx=4096 + 5, top_k=32, calib_rows=1024)
+    dw = DW.build(wl, 1, W.SCOPE_KV_HEAD, walk_steps=1, reserve_bytes=1 << 30)
+    ws = rt.alloc_workspace(dw.shape)
+    for l in range(wl.layers):
+        kv.kvswap_project_keys(dw.shape, dw.K[l], dw.proj[l], dw.meta[l], 0, wl.n_ctx, ws)
+    q = dw.q_walk[0]
+    out, lse, idx, nsel = _step_buffers(dw)
+    layers = dw.layer_tables()
+    kv.kvswap_decode_step(dw.shape, layers, q, out, lse, idx, nsel, ws)
+    torch.cuda.synchronize()
+    want = (out.clone(), lse.clone(), idx.clone(), nsel.clone())
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        kv.kvswap_decode_step(dw.shape, layers, q, out, lse, idx, nsel, ws, stream=side)
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            kv.kvswap_decode_step(dw.shape, layers, q, out, lse, idx, nsel, ws, stream=side)
+    torch.cuda.synchronize()
+    for t in (out, lse):
+        t.fill_(float("nan"))
+    idx.fill_(-7)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert kv.kvswap_read_device_status(ws) == 0
+    for got, ref in zip((out, lse, idx, nsel), want):
+        assert torch.equal(got, ref)
