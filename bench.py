@@ -1,16 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the KVSwap decode hot path (predictor + sparse decode attention) on B200.
 
-A *step* is one decode step over all L layers of the workload: per layer, kvswap_score_select
-(low-rank scoring -> head sum -> group max -> top-k) followed by kvswap_sparse_decode (gather +
-split-K online-softmax attention + combine), on one stream, through the C ABI.
+A *step* is one decode step over all L layers of the workload through kvswap_decode_step: per
+layer the predictor (low-rank scoring -> head sum -> group max -> top-k) and the sparse decode
+attention (gather + split-K online-softmax attention + combine); the predictor's kernels run on
+the library's internal stream ahead of the attention's, as the paper's runtime overlaps them.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 5] [--meta joint|per_head]
     python bench.py --impl reference ...      # the CPU oracle timed on the host cores
 
 Prints ONE JSON line (rank 0).  `value` is decode steps/s with every input resident in HBM;
 `e2e` is the same step driven through kvswap_decode_step_host with the step's queries in pinned
-host memory and its outputs read back, both copies inside the timed region.
+host memory and its outputs read back, both copies inside the timed region.  Beside them:
+`roofline` (the attention call against the measured HBM peak), `roofline_score_select`,
+`schedule.lookahead_1` (the predictor held one layer ahead), `growing_context` (a token appended
+per layer before every step), `reuse_buffer` (hit rate and phase costs with the slow tier in
+pinned host memory, and the tiered step), `prefill`, `cpu_baseline`.
 """
 from __future__ import annotations
 
