@@ -132,11 +132,36 @@ def select(R: np.ndarray, M: int) -> np.ndarray:
     return idx
 
 
-def score_select(q, proj, meta, G, M, scope="kv_head"):
-    """O2..O6 chained.  Returns (idx [B,S,M'], R [B,S,NG])."""
+def score_select(q, proj, meta, G, M, scope="kv_head", head_softmax=False):
+    """O2..O6 chained.  Returns (idx [B,S,M'], R [B,S,NG]).  With head_softmax the per-head scores
+    pass through `softmax_over_context` before the head sum (the other reading of "attention
+    scores" in Sec. 4.3)."""
     Hkv = proj.shape[0]
-    R = pool(aggregate(head_scores(lowrank_query(q, proj), meta, Hkv), Hkv, scope), G)
+    s = head_scores(lowrank_query(q, proj), meta, Hkv)
+    if head_softmax:
+        s = softmax_over_context(s, q.shape[2], G)
+    R = pool(aggregate(s, Hkv, scope), G)
     return select(R, M), R
+
+
+# ------------------------------------------------------------------------------------------
+# O3'  variant: approximate attention weights instead of approximate logits
+# ------------------------------------------------------------------------------------------
+def softmax_over_context(s: np.ndarray, d: int, G: int) -> np.ndarray:
+    """p[b,h,n] = softmax_n(s[b,h,n] / sqrt(d)) over the tokens of the complete groups,
+    n < floor(N/G) G -- the weights exact attention would give them if the low-rank logits were
+    exact and nothing else were attended.  Tokens of the open group keep no weight (0); they
+    are dropped by `pool` anyway."""
+    B, Hq, N = s.shape
+    n_scored = (N // G) * G
+    p = np.zeros_like(s, dtype=np.float64)
+    if n_scored == 0:
+        return p
+    z = s[:, :, :n_scored].astype(np.float64) / np.sqrt(d)
+    z = z - z.max(axis=2, keepdims=True)
+    e = np.exp(z)
+    p[:, :, :n_scored] = e / e.sum(axis=2, keepdims=True)
+    return p
 
 
 # ------------------------------------------------------------------------------------------

@@ -663,3 +663,46 @@ def test_planted_mistakes_in_the_reuse_buffer_are_caught(monkeypatch):
     assert fails(test_reuse_buffer_hand_worked_fifo_trace)
     monkeypatch.setattr(O, "reuse_step", real)
 
+
+# ------------------------------------------------------------------------------------------
+# O3'  per-head softmax over the context (predictor variant)
+# ------------------------------------------------------------------------------------------
+def test_head_softmax_closed_form_and_normalisation():
+    """d = 4, logits 0, 2 ln 2, 2 ln 3 (so logit / sqrt(d) = 0, ln 2, ln 3): weights 1/6, 2/6, 3/6; the
+    token of the open group (N = 4, G = 3) gets none, whatever its logit."""
+    s = np.array([[[0.0, 2 * math.log(2), 2 * math.log(3), 50.0]]])
+    p = O.softmax_over_context(s, 4, 3)
+    assert np.allclose(p[0, 0], [1 / 6, 2 / 6, 3 / 6, 0.0], atol=1e-15)
+    rng = np.random.default_rng(8)
+    s = rng.normal(size=(2, 5, 23)) * 30
+    p = O.softmax_over_context(s, 64, 4)
+    assert np.allclose(p[:, :, :20].sum(axis=2), 1.0, atol=1e-12) and np.all(p[:, :, 20:] == 0)
+    assert np.allclose(O.softmax_over_context(s + 1234.5, 64, 4), p, atol=1e-12)      # shift invariance
+    import scipy.special
+    assert np.allclose(p[:, :, :20], scipy.special.softmax(s[:, :, :20] / 8.0, axis=2), atol=1e-14)
+
+
+def test_head_softmax_changes_the_ranking_only_across_heads():
+    """One head: softmax is monotone, so the selection equals the raw-logit selection.  Two heads: a
+    sharply peaked head outvotes a nearly flat one, which the raw sum does not show -- an example,
+    worked by hand, where the two readings select different groups."""
+    rng = np.random.default_rng(3)
+    proj = np.eye(4)[None]
+    meta = _dyadic(rng, (1, 1, 24, 4))
+    q1 = _dyadic(rng, (1, 1, 4))
+    a, _ = O.score_select(q1, proj, meta, 2, 3)
+    b, _ = O.score_select(q1, proj, meta, 2, 3, head_softmax=True)
+    assert np.array_equal(a, b)
+    # d = 4 (scale 1/2), G = 1, M = 1; head 0 sees logits (8, 0, 0, 0), head 1 sees (0, 10, 9.75, 9.75)
+    meta = np.zeros((1, 1, 4, 4))
+    meta[0, 0, :, 0] = [8, 0, 0, 0]
+    meta[0, 0, :, 1] = [0, 10, 9.75, 9.75]
+    q2 = np.zeros((1, 2, 4)); q2[0, 0, 0] = 1.0; q2[0, 1, 1] = 1.0
+    raw, R_raw = O.score_select(q2, proj, meta, 1, 1)
+    assert np.array_equal(R_raw[0, 0], [8, 10, 9.75, 9.75]) and raw[0, 0, 0] == 1
+    soft, R_soft = O.score_select(q2, proj, meta, 1, 1, head_softmax=True)
+    z0 = math.exp(4) + 3
+    z1 = 1 + math.exp(5) + 2 * math.exp(4.875)
+    want = [math.exp(4) / z0 + 1 / z1, 1 / z0 + math.exp(5) / z1, 1 / z0 + math.exp(4.875) / z1,
+            1 / z0 + math.exp(4.875) / z1]
+    assert np.allclose(R_soft[0, 0], want, atol=1e-14) and soft[0, 0, 0] == 0
