@@ -73,8 +73,15 @@ typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_sco
  *       in between.  The first kernel of the call then starts while the previous kernel of the
  *       stream is still finishing (programmatic dependent launch) and only waits for it before
  *       writing its own results.  Without the flag it waits first.  Results are the same.
+ *   KVSWAP_SCORE_SOFTMAX   a variant of the predictor (kvswap_score_select, and the steps built on
+ *       it): each query head's low-rank scores pass through a softmax over the tokens of the
+ *       context's complete groups, scaled by 1/sqrt(d), BEFORE the sum over heads -- the scores
+ *       of Sec. 4.3 read as attention weights rather than logits (for one head the selection is
+ *       the same; across heads a sharply peaked head then outweighs a flat one).  Group scores
+ *       lie in [0, heads per scope].  Runs on general fp32 kernels (two passes over the
+ *       metadata).  KVSWAP_ERR_UNSUPPORTED if H_q * (r + 2) floats exceed 160 KB.
  */
-enum { KVSWAP_INPUTS_SETTLED = 1 };
+enum { KVSWAP_INPUTS_SETTLED = 1, KVSWAP_SCORE_SOFTMAX = 2 };
 
 /*
  * Problem description shared by all calls.
@@ -89,7 +96,7 @@ typedef struct {
   int32_t batch, n_ctx, n_q_heads, n_kv_heads, head_dim; /* B, N, H_q, H_kv, d            */
   int32_t rank, meta_heads, group_size, top_k;           /* r, H_m in {1, H_kv}, G, M     */
   int32_t kv_dtype, meta_dtype, q_dtype, scope;          /* enums above                   */
-  int32_t flags;                                         /* 0 or KVSWAP_INPUTS_SETTLED    */
+  int32_t flags;                                         /* bit set of the flags above    */
   int64_t kv_stride_b, kv_stride_h, kv_stride_n;
   int64_t meta_stride_b, meta_stride_h, meta_stride_n;
 } kvswap_shape;

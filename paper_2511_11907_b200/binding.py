@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_PKG, "libkvswap.so")
 KVSWAP_F32, KVSWAP_BF16, KVSWAP_F16 = 0, 1, 2
 KVSWAP_SCOPE_KV_HEAD, KVSWAP_SCOPE_ALL_HEADS = 0, 1
 KVSWAP_INPUTS_SETTLED = 1      # kvswap_shape.flags
+KVSWAP_SCORE_SOFTMAX = 2
 
 
 class KVSwapError(RuntimeError):

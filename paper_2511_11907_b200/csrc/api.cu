@@ -27,7 +27,7 @@ int resolve(const kvswap_shape* s, Problem* p) {
   if (s->n_q_heads % s->n_kv_heads != 0) return KVSWAP_ERR_SHAPE;
   if (s->meta_heads != 1 && s->meta_heads != s->n_kv_heads) return KVSWAP_ERR_SHAPE;
   if (s->scope != KVSWAP_SCOPE_KV_HEAD && s->scope != KVSWAP_SCOPE_ALL_HEADS) return KVSWAP_ERR_SHAPE;
-  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED)) != 0) return KVSWAP_ERR_SHAPE;
+  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED | KVSWAP_SCORE_SOFTMAX)) != 0) return KVSWAP_ERR_SHAPE;
   if (s->n_ctx > (1 << 30) || s->batch > 65535 || s->n_q_heads > 4096) return KVSWAP_ERR_SHAPE;
   const int ekv = dtype_bytes(s->kv_dtype), em = dtype_bytes(s->meta_dtype), eq = dtype_bytes(s->q_dtype);
   if (ekv == 0 || em == 0 || eq == 0) return KVSWAP_ERR_DTYPE;
@@ -61,6 +61,7 @@ int resolve(const kvswap_shape* s, Problem* p) {
   p->Mp = std::min(p->M, p->NG);
   p->Su = (p->Hm == 1) ? p->S : p->Hkv;
   p->score_pitch = p->NG;
+  if ((p->flags & KVSWAP_SCORE_SOFTMAX) && !score_softmax_supported(*p)) return KVSWAP_ERR_UNSUPPORTED;
   return KVSWAP_OK;
 }
 
@@ -75,6 +76,7 @@ void plan_workspace(const Problem& p, Workspace* w) {
   w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
   w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * workspace_score_pitch(p));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
+  w->off_softmax = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * (size_t(p.r) + 2 * size_t(score_softmax_chunks(p))));
   w->off_adapter = off;  off += align256(project_keys_umma_scratch_bytes(p) + 1024);   // 1 KiB: tensor-map base alignment
   w->total = off;
 }
@@ -154,8 +156,14 @@ static cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, 
   float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
   Problem p = p_in;
   p.score_pitch = group_scores_opt ? p.NG : workspace_score_pitch(p);     // a caller's buffer is dense [B, S, NG]
-  cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
-  if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
+  cudaError_t e;
+  if (p.flags & KVSWAP_SCORE_SOFTMAX) {
+    float* u_heads = reinterpret_cast<float*>(base + w.off_softmax);
+    e = launch_score_softmax(p, q, proj, meta, u_heads, u_heads + size_t(p.B) * p.Hq * p.r, scores, stream);
+  } else {
+    e = launch_lowrank_query(p, q, proj, uq, stream);
+    if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
+  }
   if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
   return e;
 }

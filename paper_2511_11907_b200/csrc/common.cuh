@@ -34,6 +34,7 @@ struct Workspace {
   size_t off_uq;       // float [B, Su, r]       summed low-rank queries
   size_t off_scores;   // float [B, S, NG]       group scores R (when the caller passes no buffer)
   size_t off_partial;  // float [B, Hq, splits, d + 2]  split-K partials (m, l, acc[d])
+  size_t off_softmax;  // float [B, Hq, r] per-head low-rank queries + [B, Hq, chunks, 2] softmax statistics (scorer variant)
   size_t off_adapter;  // bf16 [H_kv, 3 r, d]       adapter split into three bf16 pieces (project_keys on tcgen05)
   size_t total;
   int splits;          // split-K factor of sparse_decode for this shape
@@ -56,6 +57,11 @@ cudaError_t launch_project_keys_layers(const Problem& p, const void* const* K, c
 cudaError_t launch_flush_rows(const Problem& p, const void* const* K_fast, const void* const* V_fast, void* const* K_slow,
                               void* const* V_slow, int n_layers, int64_t fast_rows, int64_t fast_row0, int64_t slow_row0,
                               cudaStream_t st);
+// Softmax variant of the scorer (score_softmax.cu).
+int score_softmax_chunks(const Problem& p);
+bool score_softmax_supported(const Problem& p);
+cudaError_t launch_score_softmax(const Problem& p, const void* q, const float* proj, const void* meta, float* u,
+                                 float* stats, float* scores, cudaStream_t st);
 // Reuse buffer (reuse_buffer.cu).
 bool reuse_supported(const Problem& p, int n_slots, int max_groups);
 size_t reuse_state_words(const Problem& p, int n_slots, int max_groups);

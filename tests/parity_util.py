@@ -38,10 +38,11 @@ def project_tolerance(K, proj, meta_heads, oracle_meta, meta_dtype):
     return ulp + 2.0 ** -21 * absdot
 
 
-def check_selection(R, idx_gpu, nsel_gpu, M):
+def check_selection(R, idx_gpu, nsel_gpu, M, select_band=None):
     """The selection comparator: bit-exact group selection except inside the tie band.
     R: oracle group scores [B,S,NG]; idx_gpu [B,S,M]; nsel_gpu [B,S].  Returns #problems that had
-    more than one group inside the band."""
+    more than one group inside the band.  select_band overrides the relative width of the band."""
+    rel_band = SELECT_BAND if select_band is None else select_band
     B, S, NG = R.shape
     Mp = min(M, NG)
     ambiguous_problems = 0
@@ -56,7 +57,7 @@ def check_selection(R, idx_gpu, nsel_gpu, M):
             if Mp == 0:
                 continue
             tau = np.sort(R[b, s])[::-1][Mp - 1]
-            band = SELECT_BAND * max(abs(tau), 1e-30)
+            band = rel_band * max(abs(tau), 1e-30)
             amb = np.abs(R[b, s] - tau) <= band
             must = np.flatnonzero((R[b, s] > tau) & ~amb)
             never = np.flatnonzero((R[b, s] < tau) & ~amb)
