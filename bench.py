@@ -339,6 +339,10 @@ def run_ours(args, wl):
         shape, q0[l], dw.proj[l], dw.meta[l], idx[l], nsel[l], None, ws))
     dec_wait_ms, _ = per_call_ms(lambda l: kv.kvswap_sparse_decode(
         shape, q0[l], dw.K[l], dw.V[l], idx[l], nsel[l], out[l], None, ws))
+    # predictor variant: per-head softmax over the context before the head sum (general fp32 kernels)
+    shape_soft = shape.with_flags(kv.KVSWAP_SCORE_SOFTMAX | kv.KVSWAP_INPUTS_SETTLED)
+    soft_ms, _ = per_call_ms(lambda l: kv.kvswap_score_select(
+        shape_soft, q0[l], dw.proj[l], dw.meta[l], idx[l], nsel[l], None, ws))
 
     # ---- selection overlap between consecutive steps (Sec. 4.4.2), outside the timed region ----
     for i in range(min(8, n_walk)):
@@ -552,6 +556,9 @@ def run_ours(args, wl):
                                   "avg_ms_waiting_for_previous_kernel": sel_wait_ms,
                                   "frac_waiting_for_previous_kernel": select_bytes / sel_wait_ms / 1e6 / peak,
                                   "in_step_probe_ms": statistics.mean(select_ms)},
+        "predictor_softmax_variant": {"kernel": "kvswap_score_select with KVSWAP_SCORE_SOFTMAX", "avg_ms": soft_ms,
+                                      "frac": select_bytes / soft_ms / 1e6 / peak,
+                                      "algorithmic_bytes_per_launch": select_bytes},
         "prefill": {"project_keys_ms_all_layers": prefill_ms,
                     "keys_projected_per_sec": keys_per_step / prefill_ms * 1e3,
                     "read_gbs": L * wl.batch * wl.n_kv_heads * wl.n_ctx * wl.head_dim * esz[wl.kv_dtype] / prefill_ms / 1e6},

@@ -4,7 +4,7 @@
 // of "attention scores" in Sec. 4.3).  The sum over heads no longer commutes with the dot product,
 // so each head is scored on its own, and the normaliser needs a pass of its own:
 //   lowrank_query_heads_kernel  u[b,h,:] = q[b,h,:] A_g(h) * log2(e) / sqrt(d)      (logits in base 2)
-//   softmax_stats_kernel        per (sequence, head, chunk of 4096 tokens): running max and sum of
+//   softmax_stats_kernel        per (sequence, head, chunk of 1024 tokens): running max and sum of
 //                               2^(logit - max); also clears the group-score buffer
 //   softmax_pool_kernel         combines the chunks' statistics, recomputes the logits, sums the
 //                               heads' weights per selection scope and takes the group maximum
@@ -19,7 +19,7 @@ namespace kvswap {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kTokensPerThread = 16;
+constexpr int kTokensPerThread = 4;
 constexpr int kChunkTokens = kThreads * kTokensPerThread;     // tokens per CTA
 constexpr int kHeadBlock = 8;                                 // heads scored per pass over a row
 constexpr float kLog2e = 1.4426950408889634f;
@@ -60,8 +60,9 @@ __device__ __forceinline__ void head_logits(const Problem& p, const META_T* row,
 #pragma unroll
     for (int i = 0; i < kHeadBlock; ++i) {
       if (i < nh) {
-        const float* uh = u_s + (h0 + i) * p.r + k;           // shared memory, same address across the warp
-        s[i] = fmaf(uh[0], m[0], fmaf(uh[1], m[1], fmaf(uh[2], m[2], fmaf(uh[3], m[3], s[i]))));
+        // shared memory, same address across the warp: one 16-byte broadcast read per four products
+        const float4 uh = *reinterpret_cast<const float4*>(u_s + (h0 + i) * p.r + k);
+        s[i] = fmaf(uh.x, m[0], fmaf(uh.y, m[1], fmaf(uh.z, m[2], fmaf(uh.w, m[3], s[i]))));
       }
     }
   }
@@ -78,7 +79,7 @@ template <typename META_T>
 __global__ void __launch_bounds__(kThreads)
 softmax_stats_kernel(Problem p, const float* __restrict__ u, const META_T* __restrict__ meta, float* __restrict__ stats,
                      float* __restrict__ scores, int chunks, int n_scored) {
-  extern __shared__ float u_s[];                               // [Hq][r]
+  extern __shared__ __align__(16) float u_s[];                 // [Hq][r]
   __shared__ float red_m[kThreads / 32][kHeadBlock], red_l[kThreads / 32][kHeadBlock];
   const int chunk = blockIdx.x, b = blockIdx.y;
   for (int i = threadIdx.x; i < p.Hq * p.r; i += kThreads) u_s[i] = u[int64_t(b) * p.Hq * p.r + i];
@@ -144,7 +145,7 @@ template <typename META_T>
 __global__ void __launch_bounds__(kThreads)
 softmax_pool_kernel(Problem p, const float* __restrict__ u, const META_T* __restrict__ meta,
                     const float* __restrict__ stats, float* __restrict__ scores, int chunks, int n_scored) {
-  extern __shared__ float smem[];
+  extern __shared__ __align__(16) float smem[];
   float* u_s = smem;                                           // [Hq][r]
   float* m_s = u_s + p.Hq * p.r;                               // [Hq] maximum of the head's logits
   float* z_s = m_s + p.Hq;                                     // [Hq] 1 / sum of 2^(logit - max)
