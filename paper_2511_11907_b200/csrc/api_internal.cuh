@@ -1,0 +1,26 @@
+// Host-side helpers shared by the files that implement the C ABI (api.cu, step.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace kvswap {
+inline bool misaligned(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) != 0; }
+int dtype_bytes(int t);
+
+// Defined in api.cu.
+// Argument checks of kvswap_score_select; fills the problem and the workspace plan.
+int check_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
+                       const int32_t* group_idx, const int32_t* n_selected, const float* group_scores_opt,
+                       const void* ws, size_t ws_bytes, Problem* p, Workspace* w);
+// The launches of the predictor for one layer (arguments already checked).
+cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, const void* q,
+                                const float* proj, const void* meta, int32_t* group_idx, int32_t* n_selected,
+                                float* group_scores_opt, void* ws, cudaStream_t stream);
+// Checks shared by the append calls; on success `p` describes the grown context (N + 1 tokens).
+int resolve_grown(const kvswap_shape* shape, Problem* p);
+// Checks shared by the reuse-buffer calls.
+int resolve_reuse(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, Problem* p);
+}  // namespace kvswap
