@@ -10,8 +10,19 @@
  *   kvswap_sparse_decode  softmax attention over the selected groups plus the rolling-buffer
  *                         tail                                        (Sec. 4.4, 4.4.1, 4.4.4)
  *
- * The paper keeps the full KV cache on disk; here it is an HBM-resident tensor and "loading a
- * group" is a gather of G consecutive rows.
+ * and around them
+ *
+ *   kvswap_decode_step / _host        one decode step over all layers of a model, the predictor on
+ *                                     an internal stream ahead of the attention (Sec. 4.3, 4.4)
+ *   kvswap_append_kv / _append_step   a generated token joins the rolling buffer; a completed
+ *                                     group is flushed into the compact cache      (Sec. 4.4.1)
+ *   kvswap_reuse_* , kvswap_decode_step_tiered, kvswap_append_step_tiered
+ *                                     reuse buffer (slots, slot table, FIFO) in front of a slower
+ *                                     tier that holds the whole cache              (Sec. 4.4.2)
+ *
+ * The paper keeps the full KV cache on disk; by default here it is an HBM-resident tensor and
+ * "loading a group" is a gather of G consecutive rows; the tiered calls put it in any memory the
+ * GPU can read (pinned host memory in the tests) behind reuse buffers in HBM.
  *
  * Notation: B sequences, N cached tokens, H_q query heads, H_kv KV heads, rho = H_q / H_kv,
  * g(h) = floor(h / rho), d head dim, r metadata rank, A_g = proj[g] in R^{d x r} the row block of
@@ -23,7 +34,8 @@
  *
  * General conventions
  *  - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
- *    The library never allocates, frees or keeps device memory, and never synchronises: work is
+ *    The library never allocates, frees or keeps device memory (kvswap_decode_step creates one
+ *    stream and a set of events per device on its first call), and never synchronises: work is
  *    enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and the
  *    returned status covers host-side validation and launch errors only.
  *  - Tensors are row-major with a dense last dimension; K, V and the metadata take explicit
