@@ -90,8 +90,9 @@ typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_sco
  *       context's complete groups, scaled by 1/sqrt(d), BEFORE the sum over heads -- the scores
  *       of Sec. 4.3 read as attention weights rather than logits (for one head the selection is
  *       the same; across heads a sharply peaked head then outweighs a flat one).  Group scores
- *       lie in [0, heads per scope].  Runs on general fp32 kernels (two passes over the
- *       metadata).  KVSWAP_ERR_UNSUPPORTED if H_q * (r + 2) floats exceed 160 KB.
+ *       lie in [0, heads per scope].  Two passes over the metadata (tensor cores for joint
+ *       fp16 metadata with r = 32 and H_q <= 32, general fp32 kernels otherwise).
+ *       KVSWAP_ERR_UNSUPPORTED if H_q * (r + 2) floats exceed 160 KB.
  */
 enum { KVSWAP_INPUTS_SETTLED = 1, KVSWAP_SCORE_SOFTMAX = 2 };
 
