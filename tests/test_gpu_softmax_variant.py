@@ -94,3 +94,31 @@ def test_softmax_variant_in_the_decode_step():
     torch.cuda.synchronize()
     assert torch.equal(idx_a, idx_b) and torch.isfinite(out).all()
     assert not torch.equal(idx_raw[0], idx_a[0])              # and it is a different predictor
+
+
+def _tc(**kw):
+    """A workload on the tensor-core path of the variant: joint fp16 metadata, r = 32, H_q <= 32."""
+    base = dict(layers=1, batch=2, n_ctx=8 * 150 + 5, n_q_heads=8, n_kv_heads=2, head_dim=128, rank=32, group_size=8,
+                top_k=20, kv_dtype=W.BF16, meta_dtype=W.F16, q_dtype=W.BF16, calib_rows=512)
+    base.update(kw)
+    return W.Workload("soft-tc", 1, **base)
+
+
+@pytest.mark.parametrize("name,wl,scope", [
+    ("one_head_per_scope", _tc(n_q_heads=8, n_kv_heads=8), KV),
+    ("two_heads_per_scope", _tc(n_q_heads=16, n_kv_heads=8), KV),
+    ("eight_heads_per_scope", _tc(n_q_heads=32, n_kv_heads=4), KV),
+    ("sixteen_heads_per_scope", _tc(n_q_heads=32, n_kv_heads=2), KV),
+    ("thirty_two_heads_per_scope", _tc(n_q_heads=32, n_kv_heads=1), KV),
+    ("five_heads_per_scope", _tc(n_q_heads=10, n_kv_heads=2), KV),
+    ("three_heads_all_heads_scope", _tc(n_q_heads=24, n_kv_heads=8), ALL),
+    ("group_of_one", _tc(group_size=1, n_ctx=900, top_k=64), KV),
+    ("group_of_two", _tc(group_size=2, n_ctx=2 * 601 + 1, top_k=33), KV),
+    ("group_of_four_five_heads", _tc(group_size=4, n_q_heads=10, n_kv_heads=2, n_ctx=4 * 300 + 3), KV),
+    ("group_of_sixteen", _tc(group_size=16, n_ctx=16 * 90 + 9, top_k=11), KV),
+    ("group_of_twelve", _tc(group_size=12, n_ctx=12 * 100 + 7, top_k=11), KV),
+    ("several_chunks", _tc(batch=1, n_ctx=8 * 700 + 3, top_k=100), KV),
+    ("one_group_only", _tc(n_ctx=8, top_k=4), KV),
+], ids=lambda x: x if isinstance(x, str) else None)
+def test_softmax_variant_tensor_core_shapes(name, wl, scope):
+    _check(wl, 1, scope)
