@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """Compile libkvswap.so if it is missing or older than its sources (a no-op otherwise); the
+    tests themselves never fall back to anything else."""
+    from paper_2511_11907_b200 import build
+    build.build()
+
