@@ -280,8 +280,8 @@ typedef struct {
  *               head g's slot table; with the all-heads scope one table serves every head.
  *
  * kvswap_reuse_lookup takes a step's selection (group_idx [B, S, M], n_selected [B, S], as written
- * by kvswap_score_select; entries must be distinct, entries outside [0, floor(n_ctx / G)) are "no
- * group") and writes slot_idx [B, S, M] (the slot serving each entry, -1 for "no group"), the
+ * by kvswap_score_select; a group listed twice is loaded once and both entries get its slot; entries
+ * outside [0, floor(n_ctx / G)) are "no group") and writes slot_idx [B, S, M] (the slot serving each entry, -1 for "no group"), the
  * misses in list order as miss_group / miss_slot [B, S, M] (-1 beyond the count) and n_miss
  * [B, S]; the slot table is updated.  kvswap_reuse_fill copies each missed group's G rows of K and
  * V (of the scope's heads) from the slow tier, described by `shape`'s kv strides, into its slot.

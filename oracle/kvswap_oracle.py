@@ -232,7 +232,8 @@ def reuse_step(slot_group, head, selected):
     slot_group[c] is the group id held by slot c (-1: empty) -- the paper's slot table; `head` is
     the FIFO position: slots are filled in the order 0, 1, .., C-1, 0, .., so the slot at `head`
     holds the group that was loaded longest ago.  `selected` lists the groups the predictor chose
-    for this step (distinct; entries < 0 mean "no group" and get slot -1).  In list order: a group
+    for this step (entries < 0 mean "no group" and get slot -1; a group listed twice is loaded once,
+    by its first entry, and served to both).  In list order: a group
     found in the slot table is a hit and keeps its slot; any other group is loaded into the next
     slot in FIFO order, replacing what was there.  A slot that serves this step (a hit, or a
     group loaded earlier in the same step) is passed over by the FIFO position, since the
@@ -243,9 +244,7 @@ def reuse_step(slot_group, head, selected):
     table = [int(x) for x in slot_group]
     C = len(table)
     groups = [int(j) for j in selected if j >= 0]
-    if len(set(groups)) != len(groups):
-        raise ValueError("selected groups must be distinct")
-    if len(groups) > C:
+    if len(set(groups)) > C:
         raise ValueError("the reuse buffer must hold at least the groups of one step")
     wanted = set(groups)
     where = {g: c for c, g in enumerate(table) if g >= 0}

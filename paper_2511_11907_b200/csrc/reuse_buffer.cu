@@ -88,8 +88,20 @@ reuse_lookup_kernel(int M, int NG, int C, int max_groups, const int32_t* __restr
       if (j >= 0 && j < NG) {
         grp[e] = j;
         slot[e] = group_slot[j];
-        if (slot[e] >= 0) busy[slot[e]] = 1; else ++my_miss;
+        if (slot[e] >= 0) busy[slot[e]] = 1;
+        else atomicMin(&group_slot[j], -2 - (M - i));          // claim (< -1): of a group listed twice the first entry, with the lowest mark, loads it
       }
+    }
+  }
+  __syncthreads();
+  bool loads[kMaxPerThread];
+#pragma unroll
+  for (int e = 0; e < kMaxPerThread; ++e) {
+    loads[e] = false;
+    if (grp[e] >= 0 && slot[e] < 0) {
+      slot[e] = -1;                                            // a claim read in the first pass is not a slot
+      loads[e] = group_slot[grp[e]] == -2 - (M - (i0 + e));
+      my_miss += loads[e] ? 1 : 0;
     }
   }
   int n_miss;
@@ -117,7 +129,7 @@ reuse_lookup_kernel(int M, int NG, int C, int max_groups, const int32_t* __restr
     }
   }
   __syncthreads();
-  // n_free >= n_miss because C >= M >= hits + misses (checked on the host).
+  // n_free >= n_miss because C >= M >= hits + loads (checked on the host).
 
   // ---- serve the list ---------------------------------------------------------------------------------------
 #pragma unroll
@@ -125,7 +137,7 @@ reuse_lookup_kernel(int M, int NG, int C, int max_groups, const int32_t* __restr
     const int i = i0 + e;
     if (e < per && i < M) {
       int s = slot[e];
-      if (grp[e] >= 0 && s < 0) {
+      if (loads[e]) {
         s = victim[rank];
         const int old = slot_group[s];
         if (old >= 0) group_slot[old] = -1;                     // `old` is not selected in this step
@@ -135,6 +147,16 @@ reuse_lookup_kernel(int M, int NG, int C, int max_groups, const int32_t* __restr
         miss_slot[int64_t(prob) * M + rank] = s;
         ++rank;
       }
+      slot[e] = s;
+    }
+  }
+  __syncthreads();                                             // the loaders' table entries are in place
+#pragma unroll
+  for (int e = 0; e < kMaxPerThread; ++e) {
+    const int i = i0 + e;
+    if (e < per && i < M) {
+      int s = slot[e];
+      if (grp[e] >= 0 && s < 0) s = group_slot[grp[e]];        // a repeated entry: the slot its first entry loaded
       slot_idx[int64_t(prob) * M + i] = s;
     }
   }

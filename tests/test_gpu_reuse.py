@@ -113,6 +113,38 @@ def test_lookup_follows_the_oracle_over_a_walk(n_slots, M, NG):
     assert 0.3 < hits / total < 0.9                        # the walk keeps ~70 %: most steps mostly hit
 
 
+def test_lookup_with_repeated_and_unordered_entries():
+    """Lists as kvswap_sparse_decode accepts them: unsorted, with groups listed twice or three times."""
+    G, B, NG, M, C = 4, 2, 80, 24, 24
+    wl = W.CONFIGS[1].reduced("reuse-dup", batch=B, n_ctx=G * NG + 1, top_k=M)
+    shape = rt.shape_for(wl, 1, KV)
+    S = shape.n_scopes
+    dr = DeviceReuse(shape, C, NG)
+    rng = np.random.default_rng(77)
+    tables = [[([-1] * C, 0) for _ in range(S)] for _ in range(B)]
+    for step in range(40):
+        idx = rng.integers(0, 30 + step, size=(B, S, M)).astype(np.int32)      # many repeats, drifting range
+        idx = np.minimum(idx, NG - 1)
+        nsel = np.full((B, S), M, dtype=np.int32)
+        dr.lookup(torch.from_numpy(idx).cuda(), torch.from_numpy(nsel).cuda())
+        torch.cuda.synchronize()
+        slot_idx, mg, ms, nm = (t.cpu().numpy() for t in (dr.slot_idx, dr.miss_group, dr.miss_slot, dr.n_miss))
+        head, slot_group, group_slot = dr.tables()
+        for b in range(B):
+            for s in range(S):
+                slots, loads, table, hd = O.reuse_step(*tables[b][s], idx[b, s].tolist())
+                tables[b][s] = (table, hd)
+                assert slot_idx[b, s].tolist() == slots and nm[b, s] == len(loads)
+                assert list(zip(mg[b, s, :len(loads)].tolist(), ms[b, s, :len(loads)].tolist())) == loads
+                assert slot_group[b, s].tolist() == table and head[b, s] == hd
+                assert np.all(group_slot[b, s] >= -1)                          # no claim marks left behind
+                inverse = np.full(NG, -1)
+                for c, g in enumerate(table):
+                    if g >= 0:
+                        inverse[g] = c
+                assert np.array_equal(group_slot[b, s], inverse)
+
+
 def _tiered_attention_case(wl, meta_heads, scope, n_slots, steps):
     li = W.make_layer(wl, 0, meta_heads)
     shape = rt.shape_for(wl, meta_heads, scope)

@@ -623,8 +623,12 @@ def test_reuse_buffer_invariants_on_random_walks():
 def test_reuse_buffer_rejects_what_it_cannot_serve():
     with pytest.raises(ValueError):
         O.reuse_step([-1, -1], 0, [1, 2, 3])
-    with pytest.raises(ValueError):
-        O.reuse_step([-1, -1, -1], 0, [4, 4])
+
+
+def test_reuse_buffer_serves_a_group_listed_twice_from_one_slot():
+    """Worked by hand: 4 is loaded once, by its first entry; 9 (a hit) keeps its slot for both entries."""
+    slots, loads, table, head = O.reuse_step([5, 9, -1], 2, [4, 9, 4, 9, 7])
+    assert (slots, loads, table, head) == ([2, 1, 2, 1, 0], [(4, 2), (7, 0)], [7, 9, 4], 1)
 
 
 def test_planted_mistakes_in_the_reuse_buffer_are_caught(monkeypatch):
