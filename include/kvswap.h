@@ -44,9 +44,13 @@
  *    multiples of 16 bytes (KVSWAP_ERR_ALIGN otherwise).
  *  - Inputs must be finite.  NaN/Inf never fault but give unspecified selections/outputs.
  *  - Errors are returned, never raised: no call aborts or traps.
- *  - `ws` is caller-provided scratch of at least kvswap_workspace_bytes(shape) bytes.  Its
- *    contents are undefined between calls; calls that run concurrently on different streams
- *    need different workspaces.
+ *  - `ws` is caller-provided scratch of at least kvswap_workspace_bytes(shape) bytes, cleared once
+ *    with kvswap_workspace_init before its first use.  The predictor keeps a region at its head
+ *    (sized by B, H_kv, the scope and the metadata type alone) zero from call to call; the rest is
+ *    undefined between calls.  One workspace may serve shapes that differ in n_ctx, top_k and
+ *    flags; clear it again before using it for another batch size, head count or scope, and after
+ *    a call that returned KVSWAP_ERR_CUDA.  Calls that run concurrently on different streams need
+ *    different workspaces.
  */
 #ifndef KVSWAP_H_
 #define KVSWAP_H_
@@ -121,12 +125,14 @@ size_t kvswap_workspace_bytes(const kvswap_shape* shape);
 int kvswap_validate_shape(const kvswap_shape* shape);
 
 /*
- * Device status word.  The kernels stage K/V rows through shared memory with asynchronous copies
- * and wait for them with a bounded number of attempts; a wait that runs out (which no valid
- * input can cause) is recorded in the first word of the workspace instead of hanging the GPU.
- *   kvswap_workspace_init     clears the word (asynchronously, on `cuda_stream`).  Call it once
- *                             after allocating a workspace; a workspace that was never cleared
- *                             computes correctly but reports garbage below.
+ * Workspace set-up and the device status word.  The kernels stage K/V rows through shared memory
+ * with asynchronous copies and wait for them with a bounded number of attempts; a wait that runs
+ * out (which no valid input can cause) is recorded in the first word of the workspace instead of
+ * hanging the GPU.
+ *   kvswap_workspace_init     clears the workspace (asynchronously, on `cuda_stream`): the status
+ *                             word and the counters kvswap_score_select expects to find zero.
+ *                             Required once after allocating a workspace (see the conventions
+ *                             above); a workspace that was never cleared selects wrong groups.
  *   kvswap_read_device_status waits for `cuda_stream` to drain (the only call of the library that
  *                             synchronises), then returns KVSWAP_OK, or KVSWAP_ERR_TIMEOUT if a
  *                             kernel using `ws` has given up a wait since the word was cleared.
@@ -221,7 +227,11 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
  *    KVSWAP_ERR_STATIC_SCRATCH before anything is launched.  All five benchmark configurations
  *    fit (the largest needs about 2 MiB).
  *  - The first call on each device looks up the buffer's device address (with that device
- *    current) and caches it; make that first call outside of any stream capture.
+ *    current) and caches it for the life of the process; make that first call outside of any
+ *    stream capture, and do not call this entry point on a device after the process has reset
+ *    it (cudaDeviceReset): the cached address would be stale.
+ *  - The size check is the first check after the shape's: KVSWAP_ERR_STATIC_SCRATCH is returned
+ *    whatever the pointers are.
  *  - All calls on a device share the one buffer, and it keeps whatever the previous call left
  *    there.  Nothing in it needs clearing (each call overwrites every slot it later reads), but
  *    two calls that overlap on the GPU -- different streams, or threads -- race on it and give
@@ -289,7 +299,10 @@ typedef struct {
  * group_idx = slot_idx, a shape with n_ctx = n_slots * G + (N mod G) and the reuse store's strides.
  * Hits / (hits + misses) is the paper's reuse rate.
  *
- * Limits: n_slots >= M (else KVSWAP_ERR_SHAPE: a step's groups must fit), n_slots <= 32768 and
+ * Limits: n_slots >= M (else KVSWAP_ERR_SHAPE: a step's groups must fit); floor(n_ctx / G) <=
+ * max_groups in every call that takes max_groups, the tiered steps included (else
+ * KVSWAP_ERR_SHAPE: the tables have no entry for a group id beyond max_groups, so a context that
+ * has grown past max_groups * G + G - 1 tokens needs a larger state); n_slots <= 32768 and
  * M <= 8192 (else KVSWAP_ERR_UNSUPPORTED).  KVSWAP_ERR_WORKSPACE if state_bytes is too small.
  * All calls are asynchronous on `cuda_stream`.
  */
@@ -381,8 +394,9 @@ int kvswap_decode_step_tiered(const kvswap_shape* shape, const kvswap_layers* la
  * in kvswap_append_kv).  k_new, v_new [L, B, H_kv, d] join the rolling-buffer rows of each
  * layer's reuse store (row n_slots G + N mod G).  When the token completes a group, the group's
  * G rows are written from there to rows [N+1-G, N] of the slow tier (this call WRITES K_slow and
- * V_slow) and its compact-cache rows are built.  Of `tiers` only n_slots, K_slow, V_slow,
- * K_reuse and V_reuse are used.  Asynchronous on `cuda_stream`.
+ * V_slow) and its compact-cache rows are built.  Of `tiers` only n_slots, max_groups, K_slow,
+ * V_slow, K_reuse and V_reuse are used; KVSWAP_ERR_SHAPE if the grown context has more complete
+ * groups than a non-zero max_groups.  Asynchronous on `cuda_stream`.
  */
 int kvswap_append_step_tiered(const kvswap_shape* shape, const kvswap_layers* layers,
                               const kvswap_tiers* tiers, const void* k_new, const void* v_new,

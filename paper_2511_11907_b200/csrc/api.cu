@@ -5,6 +5,7 @@
 
 #include "api_internal.cuh"
 #include "common.cuh"
+#include "topk_keys.cuh"
 
 namespace kvswap {
 
@@ -68,10 +69,24 @@ int resolve(const kvswap_shape* s, Problem* p) {
 // that the top-k kernel can load them as vectors whatever NG is.
 static int workspace_score_pitch(const Problem& p) { return (std::max(p.NG, 1) + 31) / 32 * 32; }
 
+// Room for the leading-digit histograms (score_stream.cu, topk_select.cu) is planned from the
+// batch and head counts alone, at a fixed place in front of everything else, so that one workspace
+// keeps them zero between calls while the context grows.
+static bool hist_capable(const Problem& p) {
+  return p.meta_dtype == KVSWAP_F16 && p.r == 32 && int64_t(p.B) * p.S <= 1024;
+}
+
+// The scorer counts the leading digit of every group score's key and the TopK starts from those
+// counts (several CTAs per problem) where both kernels have that path.
+static bool counts_top_digit(const Problem& p) {
+  return !(p.flags & KVSWAP_SCORE_SOFTMAX) && hist_capable(p) && score_stream_counts_top_digit(p) && topk_parts_supported(p);
+}
+
 void plan_workspace(const Problem& p, Workspace* w) {
   plan_sparse_decode(p, w);
 
   size_t off = 256;  // first 256 bytes reserved
+  w->off_hist = off;     off += hist_capable(p) ? align256(size_t(p.B) * p.S * (sizeof(uint16_t) * kKeyTopBins + sizeof(uint32_t))) : 0;
   w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
   w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * workspace_score_pitch(p));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
@@ -99,24 +114,52 @@ int check_score_select(const kvswap_shape* shape, const void* q, const float* pr
   return KVSWAP_OK;
 }
 
-// The three launches of the predictor for one layer (arguments already checked).
-cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, const void* q, const float* proj,
-                                       const void* meta, int32_t* group_idx, int32_t* n_selected,
-                                       float* group_scores_opt, void* ws, cudaStream_t stream) {
+// The predictor of one layer in two halves (arguments already checked): the scorer, which leaves the
+// group scores (and, where that path exists, the leading-digit histograms) in the workspace or the
+// caller's buffer, and the TopK over them.  A step may put other work between the two.
+cudaError_t score_launch(const Problem& p_in, const Workspace& w, const void* q, const float* proj, const void* meta,
+                         float* group_scores_opt, void* ws, cudaStream_t stream) {
   char* base = static_cast<char*>(ws);
   float* uq = reinterpret_cast<float*>(base + w.off_uq);
   float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
   Problem p = p_in;
   p.score_pitch = group_scores_opt ? p.NG : workspace_score_pitch(p);     // a caller's buffer is dense [B, S, NG]
-  cudaError_t e;
   if (p.flags & KVSWAP_SCORE_SOFTMAX) {
     float* u_heads = reinterpret_cast<float*>(base + w.off_softmax);
-    e = launch_score_softmax(p, q, proj, meta, u_heads, u_heads + size_t(p.B) * p.Hq * p.r, scores, stream);
-  } else {
-    e = launch_lowrank_query(p, q, proj, uq, stream);
-    if (e == cudaSuccess && p.NG > 0) e = launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
+    return launch_score_softmax(p, q, proj, meta, u_heads, u_heads + size_t(p.B) * p.Hq * p.r, scores, stream);
   }
-  if (e == cudaSuccess) e = launch_topk_select(p, scores, group_idx, n_selected, stream);
+  if (p.NG < 1) return cudaSuccess;                                       // nothing to score
+  if (score_stream_supported(p)) {
+    // fp16 metadata rows of 64 bytes: the tensor-core scorer, which builds the low-rank queries itself
+    // where it can and counts the leading digits of its scores for the TopK that follows
+    uint32_t* top_hist = counts_top_digit(p) ? reinterpret_cast<uint32_t*>(base + w.off_hist) : nullptr;
+    const bool fused = score_stream_fuses_query(p);
+    cudaError_t e = fused ? cudaSuccess : launch_lowrank_query(p, q, proj, uq, stream);
+    if (e != cudaSuccess) return e;
+    return launch_score_stream(p, fused ? q : nullptr, proj, uq, meta, scores, top_hist, static_cast<uint32_t*>(ws),
+                               stream);
+  }
+  cudaError_t e = launch_lowrank_query(p, q, proj, uq, stream);
+  if (e != cudaSuccess) return e;
+  return launch_score_pool(p, uq, meta, scores, static_cast<uint32_t*>(ws), stream);
+}
+
+cudaError_t select_launch(const Problem& p_in, const Workspace& w, int32_t* group_idx, int32_t* n_selected,
+                          float* group_scores_opt, void* ws, cudaStream_t stream) {
+  char* base = static_cast<char*>(ws);
+  float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
+  Problem p = p_in;
+  p.score_pitch = group_scores_opt ? p.NG : workspace_score_pitch(p);
+  if (p.NG > 0 && score_stream_supported(p) && counts_top_digit(p))
+    return launch_topk_parts(p, scores, reinterpret_cast<uint32_t*>(base + w.off_hist), group_idx, n_selected, stream);
+  return launch_topk_select(p, scores, group_idx, n_selected, stream);
+}
+
+cudaError_t score_select_launch(const Problem& p, const Workspace& w, const void* q, const float* proj,
+                                const void* meta, int32_t* group_idx, int32_t* n_selected, float* group_scores_opt,
+                                void* ws, cudaStream_t stream) {
+  cudaError_t e = score_launch(p, w, q, proj, meta, group_scores_opt, ws, stream);
+  if (e == cudaSuccess) e = select_launch(p, w, group_idx, n_selected, group_scores_opt, ws, stream);
   return e;
 }
 
@@ -138,8 +181,12 @@ int resolve_grown(const kvswap_shape* shape, Problem* p) {
 int resolve_reuse(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, Problem* p) {
   int st = resolve(shape, p);
   if (st != KVSWAP_OK) return st;
-  if (n_slots < 1 || max_groups < 1 || n_slots < p->M) return KVSWAP_ERR_SHAPE;
-  if (!reuse_supported(*p, n_slots, max_groups)) return KVSWAP_ERR_UNSUPPORTED;
+  // max_groups = 0: a call that does not touch the slot tables (the miss gather, size queries)
+  if (n_slots < 1 || max_groups < 0 || n_slots < p->M) return KVSWAP_ERR_SHAPE;
+  // The tables have one entry per group id below max_groups: a context with more complete groups
+  // than that could select a group the tables cannot record.
+  if (max_groups > 0 && p->NG > max_groups) return KVSWAP_ERR_SHAPE;
+  if (!reuse_supported(*p, n_slots, std::max(max_groups, 1))) return KVSWAP_ERR_UNSUPPORTED;
   return KVSWAP_OK;
 }
 
@@ -211,13 +258,14 @@ int kvswap_append_kv(const kvswap_shape* shape, const void* k_new, const void* v
 
 size_t kvswap_reuse_state_bytes(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups) {
   Problem p;
-  if (resolve_reuse(shape, n_slots, max_groups, &p) != KVSWAP_OK) return 0;
+  if (max_groups < 1 || resolve_reuse(shape, n_slots, max_groups, &p) != KVSWAP_OK) return 0;
   return sizeof(int32_t) * reuse_state_words(p, n_slots, max_groups);
 }
 
 int kvswap_reuse_init(const kvswap_shape* shape, int32_t n_slots, int32_t max_groups, void* state, size_t state_bytes,
                       void* cuda_stream) {
   Problem p;
+  if (max_groups < 1) return KVSWAP_ERR_SHAPE;
   int st = resolve_reuse(shape, n_slots, max_groups, &p);
   if (st != KVSWAP_OK) return st;
   if (state == nullptr) return KVSWAP_ERR_NULL;
@@ -232,6 +280,7 @@ int kvswap_reuse_lookup(const kvswap_shape* shape, int32_t n_slots, int32_t max_
                         const int32_t* n_selected, void* state, size_t state_bytes, int32_t* slot_idx,
                         int32_t* miss_group, int32_t* miss_slot, int32_t* n_miss, void* cuda_stream) {
   Problem p;
+  if (max_groups < 1) return KVSWAP_ERR_SHAPE;
   int st = resolve_reuse(shape, n_slots, max_groups, &p);
   if (st != KVSWAP_OK) return st;
   if (group_idx == nullptr || n_selected == nullptr || state == nullptr || slot_idx == nullptr ||
@@ -250,7 +299,7 @@ int kvswap_reuse_fill(const kvswap_shape* shape, int32_t n_slots, const void* K_
                       void* K_reuse, void* V_reuse, const int32_t* miss_group, const int32_t* miss_slot,
                       const int32_t* n_miss, void* cuda_stream) {
   Problem p;
-  int st = resolve_reuse(shape, n_slots, 1, &p);
+  int st = resolve_reuse(shape, n_slots, 0, &p);
   if (st != KVSWAP_OK) return st;
   if (K_slow == nullptr || V_slow == nullptr || K_reuse == nullptr || V_reuse == nullptr || miss_group == nullptr ||
       miss_slot == nullptr || n_miss == nullptr)
@@ -298,8 +347,9 @@ int kvswap_sparse_decode(const kvswap_shape* shape, const void* q, const void* K
 int kvswap_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
   if (ws == nullptr) return KVSWAP_ERR_NULL;
   if (ws_bytes < 256) return KVSWAP_ERR_WORKSPACE;
-  return cudaMemsetAsync(ws, 0, 256, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? KVSWAP_OK
-                                                                                             : KVSWAP_ERR_CUDA;
+  // The status word and the predictor's histograms must start at zero; the rest does not care.
+  return cudaMemsetAsync(ws, 0, ws_bytes, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? KVSWAP_OK
+                                                                                                  : KVSWAP_ERR_CUDA;
 }
 
 int kvswap_read_device_status(const void* ws, void* cuda_stream) {

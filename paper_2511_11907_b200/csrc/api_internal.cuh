@@ -15,7 +15,12 @@ int dtype_bytes(int t);
 int check_score_select(const kvswap_shape* shape, const void* q, const float* proj, const void* meta,
                        const int32_t* group_idx, const int32_t* n_selected, const float* group_scores_opt,
                        const void* ws, size_t ws_bytes, Problem* p, Workspace* w);
-// The launches of the predictor for one layer (arguments already checked).
+// The predictor of one layer in two halves (arguments already checked): scorer, then TopK.
+cudaError_t score_launch(const Problem& p_in, const Workspace& w, const void* q, const float* proj, const void* meta,
+                         float* group_scores_opt, void* ws, cudaStream_t stream);
+cudaError_t select_launch(const Problem& p_in, const Workspace& w, int32_t* group_idx, int32_t* n_selected,
+                          float* group_scores_opt, void* ws, cudaStream_t stream);
+// Both halves back to back.
 cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, const void* q,
                                 const float* proj, const void* meta, int32_t* group_idx, int32_t* n_selected,
                                 float* group_scores_opt, void* ws, cudaStream_t stream);

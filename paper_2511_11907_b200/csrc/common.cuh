@@ -33,6 +33,7 @@ struct Problem {
 struct Workspace {
   size_t off_uq;       // float [B, Su, r]       summed low-rank queries
   size_t off_scores;   // float [B, S, NG]       group scores R (when the caller passes no buffer)
+  size_t off_hist;     // uint16 [B, S, 4096] + uint32 [B, S]  leading-digit histograms of the group scores' keys and tickets, zero between calls
   size_t off_partial;  // float [B, Hq, splits, d + 2]  split-K partials (m, l, acc[d])
   size_t off_softmax;  // float [B, Hq, r] per-head low-rank queries + [B, Hq, chunks, 2] softmax statistics (scorer variant)
   size_t off_adapter;  // bf16 [H_kv, 3 r, d]       adapter split into three bf16 pieces (project_keys on tcgen05)
@@ -79,8 +80,23 @@ cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* p
                                  cudaStream_t st);
 cudaError_t launch_score_pool(const Problem& p, const float* uq, const void* meta, float* scores,
                               uint32_t* err, cudaStream_t st);
+// The streaming tensor-core scorer (score_stream.cu) for fp16 metadata rows of 64 bytes.  Where it
+// builds the low-rank queries itself it takes q and proj (uq unused), else uq from
+// launch_lowrank_query.  `top_hist` (may be NULL): per (sequence, scope) a histogram of the leading
+// 12 bits of the group scores' keys (4096 16-bit counters, two per word) followed, after all
+// histograms, by one ticket word per (sequence, scope).  Everything is zero on entry; the scorer
+// counts, and launch_topk_parts, which starts from the counts, leaves everything zero again.
+bool score_stream_supported(const Problem& p);
+bool score_stream_fuses_query(const Problem& p);
+bool score_stream_counts_top_digit(const Problem& p);
+cudaError_t launch_score_stream(const Problem& p, const void* q, const float* proj, const float* uq,
+                                const void* meta, float* scores, uint32_t* top_hist, uint32_t* err,
+                                cudaStream_t st);
 cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* group_idx,
                                int32_t* n_selected, cudaStream_t st);
+bool topk_parts_supported(const Problem& p);   // false: row too long for launch_topk_parts
+cudaError_t launch_topk_parts(const Problem& p, const float* scores, uint32_t* top_hist,
+                              int32_t* group_idx, int32_t* n_selected, cudaStream_t st);
 cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K,
                                  const void* V, const int32_t* group_idx, const int32_t* n_selected,
                                  float* partial, float* out, float* lse, uint32_t* err, cudaStream_t st);

@@ -8,11 +8,12 @@
 //   per-head metadata, KV_HEAD:    one term, head g = s, uq row g = u_g;
 //   per-head metadata, ALL_HEADS:  H_kv terms, term t reads head t with uq row t = u_t.
 //
-// Two scorers:
-//   score_pool_tiles_kernel  the streaming path for 64-byte metadata rows (r = 32 fp16 or r = 16
-//                            fp32) that are dense in memory, G a power of two <= 32 and one
-//                            term per score.  Warps pull 2 KB tiles of 32 rows into shared memory
-//                            with bulk asynchronous copies, several tiles in flight per warp.
+// The scorers of this file (fp16 metadata rows of 64 bytes take the tensor-core scorer of
+// score_stream.cu, which also builds the low-rank queries itself):
+//   score_pool_tiles_kernel  the streaming path for fp32 metadata rows of 64 bytes (r = 16) that
+//                            are dense in memory, G a power of two <= 32 and one term per score.
+//                            Warps pull 2 KB tiles of 32 rows into shared memory with bulk
+//                            asynchronous copies, several tiles in flight per warp.
 //   score_pool_kernel        every other shape (any r, G, stride; the H_kv-term case).
 #include <algorithm>
 
@@ -315,213 +316,6 @@ score_pool_tiles_kernel(Problem p, const float* __restrict__ uq, const META_T* _
 }
 
 // ------------------------------------------------------------------------------------------
-// K2, streaming path for joint fp16 metadata scored for several scopes at once.
-//
-// With one metadata row feeding up to 8 scores (the per-KV-head scopes of the joint adapter) the
-// work per row is an [rows x 32] . [32 x 8] contraction at 8 FLOP per byte, which the fp32 pipes
-// cannot sustain at HBM rate; it runs on the tensor cores instead (mma.sync m16n8k16, fp16 inputs,
-// fp32 accumulation), 16 rows per instruction group.  The summed low-rank queries stay fp32-exact:
-// each is scaled by a power of two and split into an fp16 head and an fp16 remainder (two
-// products per k-step), so the only rounding is the accumulator's.
-//
-// Operand layout.  A 16-byte shared-memory read gives lane (g = lane / 4, t = lane % 4) the rank
-// entries 8t..8t+7 of row g of an 8-row block.  The contraction index may be permuted freely as
-// long as both operands agree, so k-step j takes entries 8t+4j..8t+4j+3 as the four values the
-// lane owes for token g (the column operand, 8 tokens wide), and the row operand holds the same
-// entries of the query of scope g (rows 8..15 are zero).  The accumulator then holds, in lane
-// (g, t), the scores of scope g for tokens 2t and 2t+1.
-// ------------------------------------------------------------------------------------------
-__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                         uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ uint32_t pack_half2(__half lo, __half hi) {
-  return uint32_t(__half_as_ushort(lo)) | (uint32_t(__half_as_ushort(hi)) << 16);
-}
-
-template <int GS>                                    // GS = log2(G), 0..5
-__global__ void __launch_bounds__(kWarps * 32, 3)
-score_pool_mma_kernel(Problem p, const float* __restrict__ uq, const __half* __restrict__ meta,
-                      float* __restrict__ scores, int tiles_per_row, int n_sub,
-                      uint32_t* __restrict__ err) {
-  constexpr int g_shift = GS;
-  constexpr int NS = 8;
-  extern __shared__ __align__(128) unsigned char dyn[];
-  unsigned char* tiles = dyn;
-  TileControl* ctl = reinterpret_cast<TileControl*>(dyn + kWarps * kDepth * kTileBytes);
-  float* outbuf = reinterpret_cast<float*>(dyn + kWarps * kDepth * kTileBytes + sizeof(TileControl));
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rq = lane >> 2, qt = lane & 3;
-  if (lane == 0) {                                  // every warp sets up its own stages: no CTA-wide wait
-    for (int s = 0; s < kDepth; ++s) mbar_init(smem_addr(&ctl->full[warp * kDepth + s]), 1);
-    mbar_init_fence();
-  }
-  __syncwarp();
-
-  const int rows_total = p.NG * p.G;
-  const int hm_count = (p.Hm == 1) ? 1 : p.Hkv;   // per-head metadata: one scope (column 0) per head
-  const int64_t items = int64_t(p.B) * hm_count * n_sub * tiles_per_row;
-  const int64_t gw = int64_t(blockIdx.x) * kWarps + warp, n_gw = int64_t(gridDim.x) * kWarps;
-  const int first = int(items * gw / n_gw), last = int(items * (gw + 1) / n_gw);
-  const int my_tiles = last - first;
-  int f_tile = first % tiles_per_row, f_rest = first / tiles_per_row;     // rest = (b * hm_count + hm) * n_sub + sub
-  int c_tile = f_tile, c_rest = f_rest;
-
-  const uint32_t ring = smem_addr(tiles) + uint32_t(warp) * kDepth * kTileBytes;
-  const __half* f_base = nullptr;                   // metadata of the fill cursor's (sequence, head)
-  int f_base_rest = -1;
-  auto fill = [&](int stage) {
-    if (lane == 0) {
-      if (f_rest != f_base_rest) {                  // divisions only when the cursor enters a new row set
-        f_base_rest = f_rest;
-        const int bh = f_rest / n_sub;
-        f_base = meta + int64_t(bh / hm_count) * p.meta_sb + int64_t(bh % hm_count) * p.meta_sh;
-      }
-      const int rows = min(kTileRows, rows_total - f_tile * kTileRows);
-      const uint32_t bar = smem_addr(&ctl->full[warp * kDepth + stage]);
-      mbar_arrive_expect_tx(bar, uint32_t(rows) * kRowBytes);
-      bulk_g2s(ring + uint32_t(stage) * kTileBytes, f_base + int64_t(f_tile) * kTileRows * p.meta_sn,
-               uint32_t(rows) * kRowBytes, bar);
-    }
-    if (++f_tile == tiles_per_row) { f_tile = 0; ++f_rest; }
-  };
-  // The metadata is never written by the kernel that precedes this one in the same call.
-  for (int k = 0; k < kDepth && k < my_tiles; ++k) fill(k);
-  pdl_wait();
-  pdl_trigger();
-
-  uint32_t bhi[2][2], blo[2][2];                    // query fragments (head, remainder) of k-steps 0 and 1
-  float inv = 1.f;                                  // undoes the scaling of this lane's scope
-  int cur_rest = -1, b = 0, sub = 0, hm = 0;
-  float* out_row0 = scores;                         // scores row of the first scope of the current block
-  int ns_cur = 1;
-  constexpr int gb = (GS < 3) ? GS : 3;             // butterfly levels over the row bits
-  float run = -INFINITY;                            // running maximum of a 16- or 32-row group
-  float* out = outbuf + warp * (NS * kOutStride);
-  int stage = 0;
-  uint32_t phase = 0;
-  bool timed_out = false;
-  for (int k = 0; k < my_tiles; ++k) {
-    const int tile = c_tile;
-    if (c_rest != cur_rest) {                       // new (sequence, scope block): rebuild B
-      cur_rest = c_rest;
-      sub = c_rest % n_sub;
-      { const int bh = c_rest / n_sub; hm = bh % hm_count; b = bh / hm_count; }
-      // this lane supplies the query of column rq: scope sub * 8 + rq (joint) or head hm (column 0 only)
-      const int urow = (p.Hm == 1) ? sub * NS + rq : hm;
-      const bool have = (p.Hm == 1) ? (urow < p.S) : (rq == 0);
-      float u[8];
-      if (have) {
-        const float4* ur = reinterpret_cast<const float4*>(uq + (int64_t(b) * p.Su + urow) * p.r + qt * 8);
-        const float4 x = ur[0], y = ur[1];
-        u[0] = x.x; u[1] = x.y; u[2] = x.z; u[3] = x.w; u[4] = y.x; u[5] = y.y; u[6] = y.z; u[7] = y.w;
-      } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) u[i] = 0.f;
-      }
-      float mx = 0.f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) mx = fmaxf(mx, fabsf(u[i]));
-      mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
-      // power of two that brings the largest entry into [2^14, 2^15)
-      int sh = 0;
-      if (mx > 0.f && mx < INFINITY) sh = min(120, max(-113, 14 - (int((__float_as_uint(mx) >> 23) & 0xffu) - 127)));
-      const float scale = __uint_as_float(uint32_t(sh + 127) << 23);
-      inv = __uint_as_float(uint32_t(127 - sh) << 23);
-      __half hi[8], lo[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float us = u[i] * scale;
-        hi[i] = __float2half_rn(us);
-        lo[i] = __float2half_rn(us - __half2float(hi[i]));
-      }
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        bhi[j][0] = pack_half2(hi[4 * j], hi[4 * j + 1]); bhi[j][1] = pack_half2(hi[4 * j + 2], hi[4 * j + 3]);
-        blo[j][0] = pack_half2(lo[4 * j], lo[4 * j + 1]); blo[j][1] = pack_half2(lo[4 * j + 2], lo[4 * j + 3]);
-      }
-      const int s0 = (p.Hm == 1) ? sub * NS : hm;
-      ns_cur = (p.Hm == 1) ? min(NS, p.S - s0) : 1;
-      out_row0 = scores + (int64_t(b) * p.S + s0) * p.score_pitch;
-    }
-    if (++c_tile == tiles_per_row) { c_tile = 0; ++c_rest; }
-    if (!__all_sync(kFull, mbar_wait(smem_addr(&ctl->full[warp * kDepth + stage]), phase))) { timed_out = true; break; }
-    const int rows = min(kTileRows, rows_total - tile * kTileRows);
-    const int ngt = rows >> g_shift;                // groups in this tile
-    const uint32_t base = ring + uint32_t(stage) * kTileBytes + uint32_t(lane) * 16u;
-    // Scopes are the row operand (rows 8..15 unused), 8 tokens the column operand: lane (g, t)
-    // receives the scores of scope g for tokens 2t and 2t+1 of each 8-row read, so a group's
-    // maximum is a max over two registers and at most two shuffles.
-    const bool scope_ok = rq < ns_cur;
-    float* orow = out + rq * kOutStride;
-#pragma unroll
-    for (int it = 0; it < kTileRows / 8; ++it) {
-      if (it * 8 < rows) {
-        uint32_t w[4];
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
-                     : "r"(base + uint32_t(it) * 8u * kRowBytes));
-        float d[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          mma16816(d, bhi[j][0], 0u, bhi[j][1], 0u, w[2 * j], w[2 * j + 1]);
-          mma16816(d, blo[j][0], 0u, blo[j][1], 0u, w[2 * j], w[2 * j + 1]);
-        }
-        const float x0 = d[0] * inv, x1 = d[1] * inv;            // tokens 2t and 2t+1 of this read
-        if constexpr (GS == 0) {
-          if (scope_ok) { orow[it * 8 + 2 * qt] = x0; orow[it * 8 + 2 * qt + 1] = x1; }
-        } else {
-          float m = fmaxf(x0, x1);
-          if constexpr (GS >= 2) m = fmaxf(m, __shfl_xor_sync(kFull, m, 1));
-          if constexpr (GS >= 3) m = fmaxf(m, __shfl_xor_sync(kFull, m, 2));
-          if constexpr (GS == 1) { if (scope_ok) orow[it * 4 + qt] = m; }
-          else if constexpr (GS == 2) { if (scope_ok && (qt & 1) == 0) orow[it * 2 + (qt >> 1)] = m; }
-          else if constexpr (GS == 3) { if (scope_ok && qt == 0) orow[it] = m; }
-          else {                                                 // G = 16 or 32: 2 or 4 reads per group
-            run = fmaxf(run, m);
-            if (((it + 1) & ((1 << (GS - 3)) - 1)) == 0) {
-              if (scope_ok && qt == 0) orow[it >> (GS - 3)] = run;
-              run = -INFINITY;
-            }
-          }
-        }
-      }
-    }
-    __syncwarp();
-    {
-      float* dst = out_row0 + ((tile * kTileRows) >> g_shift);
-      if (rows == kTileRows) {                      // full tile: 32 >> g_shift groups, a power of two
-        const int sh = 5 - g_shift;
-        for (int i = lane; i < (ns_cur << sh); i += 32) {
-          const int s = i >> sh, gi = i & ((1 << sh) - 1);
-          dst[int64_t(s) * p.score_pitch + gi] = out[s * kOutStride + gi];
-        }
-      } else {
-        for (int i = lane; i < ns_cur * ngt; i += 32) {
-          const int s = i / ngt, gi = i - s * ngt;
-          dst[int64_t(s) * p.score_pitch + gi] = out[s * kOutStride + gi];
-        }
-      }
-    }
-    __syncwarp();
-    if (k + kDepth < my_tiles) fill(stage);
-    if (++stage == kDepth) { stage = 0; phase ^= 1u; }
-  }
-  if (timed_out) {
-    if (lane == 0 && err) atomicExch(err, kDevTimeoutFull);
-    for (int s = 0; s < kDepth; ++s) {
-      mbar_wait(smem_addr(&ctl->full[warp * kDepth + s]), 0);
-      mbar_wait(smem_addr(&ctl->full[warp * kDepth + s]), 1);
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------------------
 // K2: generic fp32 scorer.  A CTA owns a tile of whole groups of one sequence and up to NS
 // scores per token that share the same metadata row.
 // ------------------------------------------------------------------------------------------
@@ -635,35 +429,6 @@ cudaError_t launch_tiles(const Problem& p, const float* uq, const void* meta, fl
                     tiles_per_row, n_sub, g_shift, err);
 }
 
-cudaError_t launch_mma(const Problem& p, const float* uq, const void* meta, float* scores, int g_shift,
-                       uint32_t* err, cudaStream_t st) {
-  constexpr int NS = 8;
-  const int rows_total = p.NG * p.G;
-  const int tiles_per_row = (rows_total + kTileRows - 1) / kTileRows;
-  const int n_sub = (p.Hm == 1) ? (p.S + NS - 1) / NS : 1;
-  const int64_t items = int64_t(p.B) * ((p.Hm == 1) ? 1 : p.Hkv) * n_sub * tiles_per_row;
-  const int64_t want = (items + kWarps - 1) / kWarps;
-  // Three CTAs per SM hide the per-tile bookkeeping better, but only pay when every warp still has
-  // a fair number of tiles; short streams run as one wave of two per SM.
-  const int per_sm = (items >= int64_t(10) * 2 * kNumSMs * kWarps) ? 3 : 2;
-  const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(per_sm * kNumSMs, want)));
-  const size_t smem = size_t(kWarps) * kDepth * kTileBytes + sizeof(TileControl) + sizeof(float) * kWarps * NS * kOutStride;
-  auto go = [&](auto kern) -> cudaError_t {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    return launch_pdl(kern, dim3(ctas), dim3(kWarps * 32), smem, st, p, uq, static_cast<const __half*>(meta), scores,
-                      tiles_per_row, n_sub, err);
-  };
-  switch (g_shift) {
-    case 0: return go(score_pool_mma_kernel<0>);
-    case 1: return go(score_pool_mma_kernel<1>);
-    case 2: return go(score_pool_mma_kernel<2>);
-    case 3: return go(score_pool_mma_kernel<3>);
-    case 4: return go(score_pool_mma_kernel<4>);
-    default: return go(score_pool_mma_kernel<5>);
-  }
-}
-
 template <typename META_T>
 cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, float* scores, uint32_t* err,
                         cudaStream_t st) {
@@ -671,15 +436,11 @@ cudaError_t launch_meta(const Problem& p, const float* uq, const void* meta, flo
   for (int s = 0; s <= 5; ++s) if ((1 << s) == p.G) g_shift = s;
   const bool one_term = (p.Hm == 1) || (p.scope == KVSWAP_SCOPE_KV_HEAD);
   const int64_t tile_items = int64_t(p.B) * p.Hkv * ((int64_t(p.NG) * p.G + kTileRows - 1) / kTileRows);
+  // fp16 rows of this kind are served by the tensor-core scorer (score_stream.cu)
   const bool streaming = one_term && g_shift >= 0 && p.r * int(sizeof(META_T)) == kRowBytes && p.meta_sn == p.r &&
                          tile_items < (int64_t(1) << 30);
-  if (streaming) {
-    // fp16 metadata: the tensor-core scorer serves every streaming case (with one score per
-    // row it uses one of its eight columns; it is still far cheaper in instructions per row
-    // than the fp32 pipes, which at one dot product per 64-byte row are issue-bound, not HBM-bound).
-    if constexpr (std::is_same<META_T, __half>::value) {
-      return launch_mma(p, uq, meta, scores, g_shift, err, st);
-    } else {
+  if constexpr (!std::is_same<META_T, __half>::value) {
+    if (streaming) {
       const int ns = (p.Hm == 1) ? p.S : 1;
       if (ns == 1) return launch_tiles<META_T, 1>(p, uq, meta, scores, g_shift, err, st);
       if (ns == 2) return launch_tiles<META_T, 2>(p, uq, meta, scores, g_shift, err, st);

@@ -24,7 +24,9 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[KVSWAP_STATIC_SCRATCH_BYTES];
 
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel could
-// use.  The device address is looked up once per device, with that device current, and cached.
+// use.  The device address is looked up once per device, with that device current, and cached
+// for the life of the process: a process that resets a device (cudaDeviceReset) must not call
+// this entry point on it afterwards, since the cached address would be stale.
 constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
 void* g_scratch_addr[kMaxDevices] = {};
@@ -57,6 +59,13 @@ extern "C" int kvswap_sparse_decode_static(const kvswap_shape* shape, const void
   Problem p;
   int st = resolve(shape, &p);
   if (st != KVSWAP_OK) return st;
+  // The size check comes first of all: a problem that cannot run here is refused whatever else
+  // is wrong with the call, before any pointer is looked at.
+  Workspace w;
+  plan_workspace(p, &w);
+  // The first 256 bytes hold the device status word, the partials follow.
+  const size_t need = 256 + sizeof(float) * size_t(p.B) * p.Hq * w.splits * (p.d + 2);
+  if (need > size_t(KVSWAP_STATIC_SCRATCH_BYTES)) return KVSWAP_ERR_STATIC_SCRATCH;
   if (q == nullptr || K == nullptr || V == nullptr || group_idx == nullptr || n_selected == nullptr ||
       out == nullptr)
     return KVSWAP_ERR_NULL;
@@ -64,11 +73,6 @@ extern "C" int kvswap_sparse_decode_static(const kvswap_shape* shape, const void
   if (mis(q, 16) || mis(K, 16) || mis(V, 16) || mis(out, 16) || mis(group_idx, 4) || mis(n_selected, 4) ||
       (lse_opt && mis(lse_opt, 4)))
     return KVSWAP_ERR_ALIGN;
-  Workspace w;
-  plan_workspace(p, &w);
-  // The first 256 bytes hold the device status word, the partials follow.
-  const size_t need = 256 + sizeof(float) * size_t(p.B) * p.Hq * w.splits * (p.d + 2);
-  if (need > size_t(KVSWAP_STATIC_SCRATCH_BYTES)) return KVSWAP_ERR_STATIC_SCRATCH;
   void* scratch = nullptr;
   if (scratch_address(&scratch) != cudaSuccess) return KVSWAP_ERR_CUDA;
   cudaError_t e = launch_sparse_decode(p, w, q, K, V, group_idx, n_selected,

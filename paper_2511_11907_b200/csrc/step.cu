@@ -129,6 +129,7 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
   size_t ws_attn_bytes = ws_bytes;
   if (tiers != nullptr) {
     Problem pr;
+    if (tiers->max_groups < 1) return KVSWAP_ERR_SHAPE;
     st = resolve_reuse(shape, tiers->n_slots, tiers->max_groups, &pr);
     if (st != KVSWAP_OK) return st;
     if (tiers->K_slow == nullptr || tiers->V_slow == nullptr || tiers->K_reuse == nullptr ||
@@ -167,7 +168,55 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
     if (misaligned(layers->proj[l]) || misaligned(layers->meta[l])) return KVSWAP_ERR_ALIGN;
   }
 
-  // Schedule (Sec. 4.3, online prediction, and Sec. 4.4): a layer's groups are predicted ahead of
+  if (tiers == nullptr) {
+    // Schedule (Sec. 4.3, online prediction, and Sec. 4.4): layer l + 1 is scored ahead of layer l's
+    // attention -- as early as a model allows whose layer-(l+1) prediction is formed from the input of
+    // layer l, which exists once layer l - 1 has been attended -- and its TopK follows that attention.
+    // All on the caller's stream, every kernel a programmatic dependent launch, so each kernel's
+    // set-up and first fetches overlap its predecessor's tail:
+    //   score(0) select(0) | score(1) attention(0) select(1) | score(2) attention(1) select(2) | ...
+    // The scorer streams the compact cache at HBM rate and the attention gathers at HBM rate; neither
+    // leaves the other room on an SM, so they run one after the other, and what the order hides is
+    // the latency-bound part: the TopK of layer l + 1 is not needed before attention l + 1, and the
+    // gather of layer l starts fetching while the scorer of layer l + 1 drains.
+    // Settled inputs: q is an input of the step; a selection is complete before the scorer that
+    // precedes its attention passes its own dependency wait.
+    Problem p_settled = p;
+    p_settled.flags |= KVSWAP_INPUTS_SETTLED;
+    kvswap_shape shape_settled = *shape;
+    shape_settled.flags |= KVSWAP_INPUTS_SETTLED;
+    auto ev = [&](void* e) { if (e != nullptr) cudaEventRecord(static_cast<cudaEvent_t>(e), stream); };
+    auto probed = [&](int l) { return probe_opt != nullptr && probe_opt->layer == l; };
+    auto score = [&](int l) -> int {
+      if (probed(l)) ev(probe_opt->ev_begin);
+      const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+      return score_launch(p_settled, w, ql, layers->proj[l], layers->meta[l], nullptr, ws, stream) == cudaSuccess
+                 ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+    };
+    auto select = [&](int l) -> int {
+      const cudaError_t e = select_launch(p_settled, w, group_idx + size_t(l) * idx_elems,
+                                          n_selected + size_t(l) * nsel_elems, nullptr, ws, stream);
+      if (probed(l)) ev(probe_opt->ev_mid);
+      return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
+    };
+    int status = score(0);
+    if (status == KVSWAP_OK) status = select(0);
+    for (int l = 0; l < L && status == KVSWAP_OK; ++l) {
+      if (l + 1 < L) status = score(l + 1);
+      if (status != KVSWAP_OK) break;
+      const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+      // (the last layer's attention follows its own TopK directly: that selection is not settled)
+      status = kvswap_sparse_decode(l + 1 < L ? &shape_settled : shape, ql, layers->K[l], layers->V[l],
+                                    group_idx + size_t(l) * idx_elems,
+                                    n_selected + size_t(l) * nsel_elems, out + size_t(l) * out_elems,
+                                    lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes, cuda_stream);
+      if (probed(l)) ev(probe_opt->ev_end);
+      if (status == KVSWAP_OK && l + 1 < L) status = select(l + 1);
+    }
+    return status;
+  }
+
+  // Tiered schedule: a layer's groups are predicted ahead of
   // its attention, concurrently with the layers before it.  The predictor therefore runs on a
   // stream of its own, ahead of the attention on the caller's stream by at most `look` layers
   // (any number when the caller sets no limit):
@@ -271,7 +320,7 @@ int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, c
 
 size_t kvswap_tiered_workspace_bytes(const kvswap_shape* shape, int32_t n_slots) {
   Problem p;
-  if (resolve_reuse(shape, n_slots, 1, &p) != KVSWAP_OK) return 0;
+  if (resolve_reuse(shape, n_slots, 0, &p) != KVSWAP_OK) return 0;
   const kvswap_shape r = reuse_store_shape(*shape, n_slots);
   const size_t tail = kvswap_workspace_bytes(&r);
   if (tail == 0) return 0;
@@ -298,6 +347,8 @@ int kvswap_append_step_tiered(const kvswap_shape* shape, const kvswap_layers* la
       tiers->V_reuse == nullptr || k_new == nullptr || v_new == nullptr)
     return KVSWAP_ERR_NULL;
   if (tiers->n_slots < 1) return KVSWAP_ERR_SHAPE;
+  // the grown context must still fit the slot tables the next tiered step will use
+  if (tiers->max_groups > 0 && p.NG > tiers->max_groups) return KVSWAP_ERR_SHAPE;
   if (misaligned(k_new) || misaligned(v_new)) return KVSWAP_ERR_ALIGN;
   const int L = layers->n_layers;
   for (int l = 0; l < L; ++l) {

@@ -149,6 +149,10 @@ def test_reuse_buffer_calls_validate_before_touching_the_gpu(lib):
                                    None) == 4
     assert lib.kvswap_reuse_lookup(ref, 64, 256, fake, fake, fake, 64, fake, fake, fake, fake, None) == 5
     assert lib.kvswap_reuse_lookup(ref, 8, 256, fake, fake, fake, 1 << 20, fake, fake, fake, fake, None) == 2
+    # the context has floor(1024 / 4) = 256 complete groups: tables sized for fewer cannot record all of them
+    assert lib.kvswap_reuse_lookup(ref, 64, 255, fake, fake, fake, 1 << 20, fake, fake, fake, fake, None) == 2
+    assert lib.kvswap_reuse_init(ref, 64, 255, fake, 1 << 20, None) == 2
+    assert kv.kvswap_reuse_state_bytes(s, 64, 255) == 0
     assert lib.kvswap_reuse_fill(ref, 64, None, fake, fake, fake, fake, fake, fake, None) == 1
     assert lib.kvswap_reuse_fill(ref, 64, ctypes.c_void_p(4100), fake, fake, fake, fake, fake, fake, None) == 4
     assert lib.kvswap_reuse_fill(ref, 8, fake, fake, fake, fake, fake, fake, fake, None) == 2
@@ -174,6 +178,8 @@ def test_tiered_step_validates_before_touching_the_gpu(lib):
     assert call(ctypes.byref(few_slots), 1 << 30) == 2
     no_out = kv.kvswap_tiers(64, 256, ptab, ptab, ptab, ptab, ptab, 1 << 20, None, 4096, 4096, 4096)
     assert call(ctypes.byref(no_out), 1 << 30) == 1
+    short_tables = kv.kvswap_tiers(64, 255, ptab, ptab, ptab, ptab, ptab, 1 << 20, 4096, 4096, 4096, 4096)
+    assert call(ctypes.byref(short_tables), 1 << 30) == 2                  # 256 complete groups, tables for 255
     # tiered append: capacity rule as for kvswap_append_kv, then the tables
     N, d, r = 1024, 64, 16
     roomy = good_shape(kv_strides=(2 * (N + 8) * d, (N + 8) * d, d), meta_strides=((N + 8) * r, (N + 8) * r, r))
@@ -182,6 +188,7 @@ def test_tiered_step_validates_before_touching_the_gpu(lib):
     assert app(roomy, None) == 1
     no_store = kv.kvswap_tiers(64, 256, ptab, ptab, None, ptab, ptab, 1 << 20, 4096, 4096, 4096, 4096)
     assert app(roomy, ctypes.byref(no_store)) == 1
+    assert app(roomy, ctypes.byref(short_tables)) == 2                     # the grown context outruns the tables
 
 
 def test_status_strings_and_version(lib):

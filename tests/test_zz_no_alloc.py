@@ -5,9 +5,10 @@ library.
 
 Checked here, through the C ABI: its output equals that of kvswap_sparse_decode (which gets a
 caller-allocated workspace) on two calls in a row with different inputs, so stale partials of
-the first call cannot leak into the second; and a problem too large for the built-in buffer is
-refused with its own status code.  The file name sorts last so that a run stopping at the first
-failure has already run every other test."""
+the first call cannot leak into the second; the device memory in use is the same before and
+after a call (the property in its name); and a problem too large for the built-in buffer is
+refused with its own status code before any pointer is looked at.  The file name sorts last so
+that a run stopping at the first failure has already run every other test."""
 import ctypes
 
 import numpy as np
@@ -58,6 +59,24 @@ def test_static_scratch_entry_matches_workspace_entry_on_two_calls_in_a_row():
         assert np.abs(got_lse - want_lse).max() <= tol, f"call {call}"
 
 
+def test_static_scratch_entry_leaves_device_memory_as_it_found_it():
+    wl = W.REDUCED[3]
+    li = W.make_layer(wl, 0, 1)
+    dl = DeviceLayer(li, W.SCOPE_KV_HEAD)
+    out, lse = rt.alloc_output(dl.shape)
+    call = lambda: kv.kvswap_sparse_decode_static(dl.shape, dl.q, dl.K, dl.V, dl.idx, dl.nsel, out, lse)
+    call()                                              # the first call on a device looks up the buffer's address
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    torch0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, "the driver reports a different amount of free device memory after the calls"
+    assert torch.cuda.memory_allocated() == torch0 and torch.cuda.memory_reserved() == reserved0
+
+
 def test_static_scratch_entry_refuses_problems_beyond_its_buffer():
     # 2048 sequences x 32 heads x 130 floats of partials = 34 MB > the 8 MiB built-in buffer.
     shape = kv.make_shape(batch=2048, n_ctx=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, rank=32,
@@ -66,7 +85,7 @@ def test_static_scratch_entry_refuses_problems_beyond_its_buffer():
     lib = kv.load()
     lib.kvswap_sparse_decode_static.restype = ctypes.c_int
     lib.kvswap_sparse_decode_static.argtypes = [ctypes.POINTER(kv.kvswap_shape)] + [ctypes.c_void_p] * 8
-    fake = ctypes.c_void_p(1 << 20)                     # aligned; the refusal comes before any launch
-    status = lib.kvswap_sparse_decode_static(ctypes.byref(shape), fake, fake, fake, fake, fake, fake, None, None)
+    # the size check precedes every pointer check, so no pointer is needed to see the refusal
+    status = lib.kvswap_sparse_decode_static(ctypes.byref(shape), None, None, None, None, None, None, None, None)
     assert status == 9
     assert "static" in kv.status_string(status)
