@@ -155,6 +155,22 @@ cudaError_t select_launch(const Problem& p_in, const Workspace& w, int32_t* grou
   return launch_topk_select(p, scores, group_idx, n_selected, stream);
 }
 
+// select_launch for problem `p_in` merged with the combine pass of a split-K attention whose gather
+// (launch_sparse_decode with combine = false, any shape) has been enqueued before: one launch.  False
+// when the select of this shape has no such kernel (the caller then launches the two separately).
+bool select_with_combine_launch(const Problem& p_in, const Workspace& w, int32_t* group_idx, int32_t* n_selected,
+                                void* ws, const float* partial, float* out, float* lse, int splits, int n_rows, int d,
+                                cudaStream_t stream, cudaError_t* result) {
+  Problem p = p_in;
+  p.score_pitch = workspace_score_pitch(p);
+  if (!(p.NG > 0 && score_stream_supported(p) && counts_top_digit(p))) return false;
+  char* base = static_cast<char*>(ws);
+  *result = launch_combine_select(p, reinterpret_cast<float*>(base + w.off_scores),
+                                  reinterpret_cast<uint32_t*>(base + w.off_hist), group_idx, n_selected, partial, out, lse,
+                                  splits, n_rows, d, stream);
+  return true;
+}
+
 cudaError_t score_select_launch(const Problem& p, const Workspace& w, const void* q, const float* proj,
                                 const void* meta, int32_t* group_idx, int32_t* n_selected, float* group_scores_opt,
                                 void* ws, cudaStream_t stream) {

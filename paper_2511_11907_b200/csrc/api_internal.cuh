@@ -20,6 +20,11 @@ cudaError_t score_launch(const Problem& p_in, const Workspace& w, const void* q,
                          float* group_scores_opt, void* ws, cudaStream_t stream);
 cudaError_t select_launch(const Problem& p_in, const Workspace& w, int32_t* group_idx, int32_t* n_selected,
                           float* group_scores_opt, void* ws, cudaStream_t stream);
+// select_launch merged with the combine pass of a split-K gather enqueued before it (one launch);
+// false when this shape's select has no such kernel.
+bool select_with_combine_launch(const Problem& p_in, const Workspace& w, int32_t* group_idx, int32_t* n_selected,
+                                void* ws, const float* partial, float* out, float* lse, int splits, int n_rows, int d,
+                                cudaStream_t stream, cudaError_t* result);
 // Both halves back to back.
 cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, const void* q,
                                 const float* proj, const void* meta, int32_t* group_idx, int32_t* n_selected,

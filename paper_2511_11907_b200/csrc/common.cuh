@@ -97,9 +97,18 @@ cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* g
 bool topk_parts_supported(const Problem& p);   // false: row too long for launch_topk_parts
 cudaError_t launch_topk_parts(const Problem& p, const float* scores, uint32_t* top_hist,
                               int32_t* group_idx, int32_t* n_selected, cudaStream_t st);
+// `combine` false: only the split-K gather runs; the caller merges the partials (launch_combine_select).
 cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K,
                                  const void* V, const int32_t* group_idx, const int32_t* n_selected,
-                                 float* partial, float* out, float* lse, uint32_t* err, cudaStream_t st);
+                                 float* partial, float* out, float* lse, uint32_t* err, cudaStream_t st,
+                                 bool combine = true);
+cudaError_t launch_combine_only(const Problem& p, const Workspace& w, const float* partial, float* out, float* lse,
+                                cudaStream_t st);
+// launch_topk_parts for problem `p` and, in the same launch, the merge of `n_rows` rows of split-K
+// partials [n_rows, splits, d + 2] (of whatever attention produced them) into out / lse.
+cudaError_t launch_combine_select(const Problem& p, const float* scores, uint32_t* top_hist, int32_t* group_idx,
+                                  int32_t* n_selected, const float* partial, float* out, float* lse, int splits,
+                                  int n_rows, int d, cudaStream_t st);
 
 // Launch with programmatic stream serialisation: the kernel may begin (up to its
 // griddepcontrol.wait) while the previous kernel in the stream is still draining.

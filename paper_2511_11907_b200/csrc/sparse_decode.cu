@@ -26,6 +26,7 @@
 #include <cstdint>
 
 #include "async_copy.cuh"
+#include "combine.cuh"
 #include "common.cuh"
 
 namespace kvswap {
@@ -562,11 +563,7 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   }
 }
 
-// K5: merge the split partials of one (sequence, head).  One CTA of D threads per row; every
-// load of the row is issued before anything is computed (one memory round trip), the split
-// weights are formed once by the first warp and shared.
-constexpr int kMaxSplits = 256;
-
+// K5: merge the split partials of one (sequence, head): one CTA of D threads per row (combine.cuh).
 template <int D>
 __global__ void __launch_bounds__(D)
 combine_kernel(const float* __restrict__ partial, float* __restrict__ out, float* __restrict__ lse, int splits) {
@@ -576,39 +573,7 @@ combine_kernel(const float* __restrict__ partial, float* __restrict__ out, float
   // partials of the gather kernel before it.
   pdl_trigger();
   pdl_wait();
-  const int64_t bh = blockIdx.x;
-  const float* src = partial + bh * splits * (D + 2);
-  const int c = threadIdx.x;
-  constexpr int kUnroll = 16;
-  float a_first[kUnroll];
-#pragma unroll
-  for (int s = 0; s < kUnroll; ++s) a_first[s] = (s < splits) ? src[s * (D + 2) + 2 + c] : 0.f;
-  if (c < 32) {
-    // weights: lane s handles splits s, s + 32, ...
-    float mx = -INFINITY;
-    for (int s = c; s < splits; s += 32) mx = fmaxf(mx, src[s * (D + 2)]);
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    float lsum = 0.f;
-    for (int s = c; s < splits; s += 32) {
-      const float w = (mx > -INFINITY) ? exp2f(src[s * (D + 2)] - mx) : 0.f;
-      w_s[s] = w;
-      lsum = fmaf(src[s * (D + 2) + 1], w, lsum);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, off);
-    if (c == 0) {
-      norm_s[0] = (lsum > 0.f) ? 1.f / lsum : 0.f;
-      norm_s[1] = (lsum > 0.f) ? (mx + log2f(lsum)) * kLn2 : -INFINITY;
-    }
-  }
-  __syncthreads();
-  float a = 0.f;
-#pragma unroll
-  for (int s = 0; s < kUnroll; ++s) if (s < splits) a = fmaf(a_first[s], w_s[s], a);
-  for (int s = kUnroll; s < splits; ++s) a = fmaf(src[s * (D + 2) + 2 + c], w_s[s], a);
-  out[bh * D + c] = a * norm_s[0];
-  if (lse != nullptr && c == 0) lse[bh] = norm_s[1];
+  combine_row<D>(partial, out, lse, splits, blockIdx.x, true, threadIdx.x, w_s, norm_s, 0);
 }
 
 template <typename KV_T, int D>
@@ -617,7 +582,7 @@ size_t stage_bytes() { return size_t(2) * kTok * D * sizeof(KV_T); }
 template <typename KV_T, typename Q_T, int D, int RH>
 cudaError_t launch_one(const Problem& p, const Workspace& w, const void* q, const void* K, const void* V,
                        const int32_t* group_idx, const int32_t* n_selected, float* partial, float* out, float* lse,
-                       uint32_t* err, cudaStream_t st) {
+                       uint32_t* err, bool combine, cudaStream_t st) {
   const int depth = w.depth;
   const size_t smem = kControlBytes + 128 + size_t(kWarps) * depth * stage_bytes<KV_T, D>();
   int g_shift = -1;
@@ -633,7 +598,7 @@ cudaError_t launch_one(const Problem& p, const Workspace& w, const void* q, cons
   e = launch_pdl(kern, dim3(w.splits, p.Hkv * (p.rho / RH), p.B), dim3(kThreads), smem, st, p,
                  static_cast<const Q_T*>(q), static_cast<const KV_T*>(K), static_cast<const KV_T*>(V), group_idx,
                  n_selected, partial, w.splits, depth, g_shift, err);
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || !combine) return e;
   return launch_pdl(combine_kernel<D>, dim3(p.B * p.Hq), dim3(D), 0, st, static_cast<const float*>(partial), out,
                     lse, w.splits);
 }
@@ -641,34 +606,34 @@ cudaError_t launch_one(const Problem& p, const Workspace& w, const void* q, cons
 template <typename KV_T, typename Q_T, int D>
 cudaError_t launch_rh(const Problem& p, const Workspace& w, const void* q, const void* K, const void* V,
                       const int32_t* gi, const int32_t* ns, float* partial, float* out, float* lse, uint32_t* err,
-                      cudaStream_t st) {
+                      bool combine, cudaStream_t st) {
   switch (w.heads_per_cta) {
-    case 8: return launch_one<KV_T, Q_T, D, 8>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    case 7: return launch_one<KV_T, Q_T, D, 7>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    case 6: return launch_one<KV_T, Q_T, D, 6>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    case 5: return launch_one<KV_T, Q_T, D, 5>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    case 4: return launch_one<KV_T, Q_T, D, 4>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    case 3: return launch_one<KV_T, Q_T, D, 3>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    case 2: return launch_one<KV_T, Q_T, D, 2>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-    default: return launch_one<KV_T, Q_T, D, 1>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
+    case 8: return launch_one<KV_T, Q_T, D, 8>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    case 7: return launch_one<KV_T, Q_T, D, 7>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    case 6: return launch_one<KV_T, Q_T, D, 6>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    case 5: return launch_one<KV_T, Q_T, D, 5>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    case 4: return launch_one<KV_T, Q_T, D, 4>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    case 3: return launch_one<KV_T, Q_T, D, 3>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    case 2: return launch_one<KV_T, Q_T, D, 2>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+    default: return launch_one<KV_T, Q_T, D, 1>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
   }
 }
 
 template <typename KV_T, typename Q_T>
 cudaError_t launch_d(const Problem& p, const Workspace& w, const void* q, const void* K, const void* V,
                      const int32_t* gi, const int32_t* ns, float* partial, float* out, float* lse, uint32_t* err,
-                     cudaStream_t st) {
-  if (p.d == 128) return launch_rh<KV_T, Q_T, 128>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-  return launch_rh<KV_T, Q_T, 64>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
+                     bool combine, cudaStream_t st) {
+  if (p.d == 128) return launch_rh<KV_T, Q_T, 128>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+  return launch_rh<KV_T, Q_T, 64>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
 }
 
 template <typename KV_T>
 cudaError_t launch_q(const Problem& p, const Workspace& w, const void* q, const void* K, const void* V,
                      const int32_t* gi, const int32_t* ns, float* partial, float* out, float* lse, uint32_t* err,
-                     cudaStream_t st) {
+                     bool combine, cudaStream_t st) {
   // q is stored as fp32 or in the K/V type (checked at validation).
-  if (p.q_dtype == KVSWAP_F32) return launch_d<KV_T, float>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
-  return launch_d<KV_T, KV_T>(p, w, q, K, V, gi, ns, partial, out, lse, err, st);
+  if (p.q_dtype == KVSWAP_F32) return launch_d<KV_T, float>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
+  return launch_d<KV_T, KV_T>(p, w, q, K, V, gi, ns, partial, out, lse, err, combine, st);
 }
 
 }  // namespace
@@ -702,13 +667,21 @@ void plan_sparse_decode(const Problem& p, Workspace* w) {
   w->depth = int(std::max<size_t>(2, std::min<size_t>(kMaxDepth, (100u << 10) / (kWarps * stage))));
 }
 
+// The combine pass alone, for a gather that was enqueued with combine = false.
+cudaError_t launch_combine_only(const Problem& p, const Workspace& w, const float* partial, float* out, float* lse,
+                                cudaStream_t st) {
+  if (p.d == 128)
+    return launch_pdl(combine_kernel<128>, dim3(p.B * p.Hq), dim3(128), 0, st, partial, out, lse, w.splits);
+  return launch_pdl(combine_kernel<64>, dim3(p.B * p.Hq), dim3(64), 0, st, partial, out, lse, w.splits);
+}
+
 cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const void* q, const void* K, const void* V,
                                  const int32_t* group_idx, const int32_t* n_selected, float* partial, float* out,
-                                 float* lse, uint32_t* err, cudaStream_t st) {
+                                 float* lse, uint32_t* err, cudaStream_t st, bool combine) {
   switch (p.kv_dtype) {
-    case KVSWAP_F32: return launch_q<float>(p, w, q, K, V, group_idx, n_selected, partial, out, lse, err, st);
-    case KVSWAP_BF16: return launch_q<__nv_bfloat16>(p, w, q, K, V, group_idx, n_selected, partial, out, lse, err, st);
-    default: return launch_q<__half>(p, w, q, K, V, group_idx, n_selected, partial, out, lse, err, st);
+    case KVSWAP_F32: return launch_q<float>(p, w, q, K, V, group_idx, n_selected, partial, out, lse, err, combine, st);
+    case KVSWAP_BF16: return launch_q<__nv_bfloat16>(p, w, q, K, V, group_idx, n_selected, partial, out, lse, err, combine, st);
+    default: return launch_q<__half>(p, w, q, K, V, group_idx, n_selected, partial, out, lse, err, combine, st);
   }
 }
 

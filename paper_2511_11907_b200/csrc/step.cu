@@ -165,10 +165,12 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
   for (int l = 0; l < L; ++l) {
     if (layers->proj[l] == nullptr || layers->meta[l] == nullptr) return KVSWAP_ERR_NULL;
     if (tiers == nullptr && (layers->K[l] == nullptr || layers->V[l] == nullptr)) return KVSWAP_ERR_NULL;
+    if (tiers == nullptr && (misaligned(layers->K[l]) || misaligned(layers->V[l]))) return KVSWAP_ERR_ALIGN;
     if (misaligned(layers->proj[l]) || misaligned(layers->meta[l])) return KVSWAP_ERR_ALIGN;
   }
 
   if (tiers == nullptr) {
+    if (misaligned(out) || (lse_opt && (reinterpret_cast<uintptr_t>(lse_opt) & 3u))) return KVSWAP_ERR_ALIGN;
     // Schedule (Sec. 4.3, online prediction, and Sec. 4.4): layer l + 1 is scored ahead of layer l's
     // attention -- as early as a model allows whose layer-(l+1) prediction is formed from the input of
     // layer l, which exists once layer l - 1 has been attended -- and its TopK follows that attention.
@@ -199,19 +201,39 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
       if (probed(l)) ev(probe_opt->ev_mid);
       return e == cudaSuccess ? KVSWAP_OK : KVSWAP_ERR_CUDA;
     };
+    // The attention of layer l and the TopK of layer l + 1: the split-K gather, then one kernel that
+    // merges its partials and selects (where the select has that form), else the two one after the other.
+    float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) + w.off_partial);
+    auto attend_then_select = [&](int l) -> int {
+      const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
+      float* out_l = out + size_t(l) * out_elems;
+      float* lse_l = lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr;
+      const int32_t* idx_l = group_idx + size_t(l) * idx_elems;
+      const int32_t* nsel_l = n_selected + size_t(l) * nsel_elems;
+      const bool next = l + 1 < L;
+      // (the last layer's attention follows its own TopK directly: that selection is not settled)
+      const Problem& pa = next ? p_settled : p;
+      if (launch_sparse_decode(pa, w, ql, layers->K[l], layers->V[l], idx_l, nsel_l, partial, out_l, lse_l,
+                               static_cast<uint32_t*>(ws), stream, /*combine=*/false) != cudaSuccess)
+        return KVSWAP_ERR_CUDA;
+      cudaError_t e = cudaSuccess;
+      const bool merged = next && select_with_combine_launch(p_settled, w, group_idx + size_t(l + 1) * idx_elems,
+                                                             n_selected + size_t(l + 1) * nsel_elems, ws, partial, out_l,
+                                                             lse_l, w.splits, p.B * p.Hq, p.d, stream, &e);
+      if (!merged) {
+        e = launch_combine_only(p, w, partial, out_l, lse_l, stream);
+      }
+      if (probed(l)) ev(probe_opt->ev_end);
+      if (e != cudaSuccess) return KVSWAP_ERR_CUDA;
+      if (next && !merged) return select(l + 1);
+      if (next && probed(l + 1)) ev(probe_opt->ev_mid);
+      return KVSWAP_OK;
+    };
     int status = score(0);
     if (status == KVSWAP_OK) status = select(0);
     for (int l = 0; l < L && status == KVSWAP_OK; ++l) {
       if (l + 1 < L) status = score(l + 1);
-      if (status != KVSWAP_OK) break;
-      const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-      // (the last layer's attention follows its own TopK directly: that selection is not settled)
-      status = kvswap_sparse_decode(l + 1 < L ? &shape_settled : shape, ql, layers->K[l], layers->V[l],
-                                    group_idx + size_t(l) * idx_elems,
-                                    n_selected + size_t(l) * nsel_elems, out + size_t(l) * out_elems,
-                                    lse_opt ? lse_opt + size_t(l) * p.B * p.Hq : nullptr, ws, ws_bytes, cuda_stream);
-      if (probed(l)) ev(probe_opt->ev_end);
-      if (status == KVSWAP_OK && l + 1 < L) status = select(l + 1);
+      if (status == KVSWAP_OK) status = attend_then_select(l);
     }
     return status;
   }
