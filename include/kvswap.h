@@ -414,6 +414,15 @@ int kvswap_decode_step_host(const kvswap_shape* shape, const kvswap_layers* laye
                             int32_t* group_idx, int32_t* n_selected, void* ws, size_t ws_bytes,
                             void* cuda_stream);
 
+/*
+ * Calibration helper of the benchmark (the paper has no counterpart): one kernel that does nothing
+ * but read `bytes` bytes at `buf` (device; both multiples of 16) with 16-byte loads, on
+ * `cuda_stream`.  Timed over buffers of the sizes the predictor and the attention stream, it gives
+ * the rate a read-only pass reaches on this GPU and, with bytes = 0, the cost of an empty launch.
+ * `sink` (device, 4 bytes, may be NULL) exists only to keep the loads alive.
+ */
+int kvswap_read_probe(const void* buf, size_t bytes, void* sink, void* cuda_stream);
+
 /* Static, NUL-terminated description of a kvswap_status value. */
 const char* kvswap_status_string(int status);
 

@@ -89,6 +89,8 @@ def load() -> ctypes.CDLL:
     lib.kvswap_workspace_init.argtypes = [V, SZ, V]
     lib.kvswap_read_device_status.restype = ctypes.c_int
     lib.kvswap_read_device_status.argtypes = [V, V]
+    lib.kvswap_read_probe.restype = ctypes.c_int
+    lib.kvswap_read_probe.argtypes = [V, SZ, V, V]
     _lib = lib
     return lib
 
@@ -195,6 +197,11 @@ def kvswap_sparse_decode(shape, q, K, V, group_idx, n_selected, out, lse_opt, ws
 def kvswap_workspace_init(ws, stream=None) -> None:
     _check(load().kvswap_workspace_init(_ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "kvswap_workspace_init")
+
+
+def kvswap_read_probe(buf, n_bytes: int, sink=None, stream=None) -> None:
+    """One read-only pass over the first n_bytes of `buf` (the benchmark's calibration kernel)."""
+    _check(load().kvswap_read_probe(_ptr(buf), int(n_bytes), _ptr(sink), _stream(stream)), "kvswap_read_probe")
 
 
 def kvswap_read_device_status(ws, stream=None) -> int:
