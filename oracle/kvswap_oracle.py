@@ -41,10 +41,52 @@ def _rho(n_q_heads: int, n_kv_heads: int) -> int:
 # ------------------------------------------------------------------------------------------
 # O1  K_lr = Flatten(K) A                                                       (Sec. 4.2)
 # ------------------------------------------------------------------------------------------
-def project_keys(K: np.ndarray, proj: np.ndarray, meta_heads: int, meta_dtype: str = "f16") -> np.ndarray:
+def e4m3_decode_table() -> np.ndarray:
+    """The 256 values of the 8-bit floating-point format E4M3 (1 sign, 4 exponent bits with bias 7,
+    3 mantissa bits; no infinities; S.1111.111 is NaN; largest finite value 448; subnormals are
+    multiples of 2^-9) -- the 8-bit storage format taken for the compact cache where the paper only
+    says that its precision can be traded (Sec. 4.1, Sec. 4.2)."""
+    vals = np.empty(256)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e, m = (code >> 3) & 0xF, code & 0x7
+        if e == 0xF and m == 0x7:
+            vals[code] = np.nan
+        elif e == 0:
+            vals[code] = sign * m * 2.0 ** -9
+        else:
+            vals[code] = sign * (8 + m) * 2.0 ** (e - 7 - 3)
+    return vals
+
+
+def e4m3_round(x: np.ndarray):
+    """Nearest E4M3 value of every entry of x (float64): round to nearest, ties to the even
+    mantissa, magnitudes beyond the largest finite value saturate to +-448.  Returns
+    (values float64, codes uint8)."""
+    x = np.asarray(x, dtype=np.float64)
+    a = np.abs(x)
+    _, ex = np.frexp(a)                                   # a = f * 2^ex, f in [0.5, 1)
+    e = np.clip(ex - 1, -6, 8)                            # binade of a, clipped to the normal range
+    quantum = np.ldexp(1.0, e - 3)                        # spacing of the format in that binade
+    quantum = np.where(a < 2.0 ** -6, 2.0 ** -9, quantum)  # subnormal spacing below the smallest normal
+    v = np.minimum(np.rint(a / quantum) * quantum, 448.0)   # np.rint rounds halves to even
+    _, ex2 = np.frexp(v)
+    e2 = np.clip(ex2 - 1, -6, 8)
+    normal = v >= 2.0 ** -6
+    mant = np.where(normal, v / np.ldexp(1.0, e2 - 3) - 8, v / 2.0 ** -9)
+    code = np.where(normal, (e2 + 7) * 8, 0) + mant
+    code = code.astype(np.int64) | np.where(np.signbit(x), 0x80, 0)
+    return np.copysign(v, x), code.astype(np.uint8)
+
+
+def project_keys(K: np.ndarray, proj: np.ndarray, meta_heads: int, meta_dtype: str = "f16",
+                 meta_exp: int = 0) -> np.ndarray:
     """Compressed K cache.  Joint: meta[b,0,n,:] = sum_g K[b,g,n,:] A_g  (Flatten is head-major,
     column g*d+c <-> K[n,g,c]).  Per-head: meta[b,g,n,:] = K[b,g,n,:] A_g.
-    The float64 result is rounded once, to nearest-even, into the storage type."""
+    The float64 result is rounded once, to nearest-even, into the storage type.  For the 8-bit
+    type "e4m3" the stored value is round(K_lr * 2^-meta_exp) (returned as float32, which holds
+    every E4M3 value exactly); the power of two only keeps the values inside the format's range
+    and is multiplied back when the metadata is scored (`score_select(..., meta_exp=)`)."""
     K64 = K.astype(np.float64)
     A = proj.astype(np.float64)
     B, Hkv, N, d = K64.shape
@@ -59,6 +101,8 @@ def project_keys(K: np.ndarray, proj: np.ndarray, meta_heads: int, meta_dtype: s
             meta[:, g] = K64[:, g] @ A[g]
     else:
         raise ValueError("meta_heads must be 1 or H_kv")
+    if meta_dtype == "e4m3":
+        return e4m3_round(np.ldexp(meta, -int(meta_exp)))[0].astype(np.float32)
     return meta.astype(_STORE[meta_dtype])
 
 
@@ -132,11 +176,14 @@ def select(R: np.ndarray, M: int) -> np.ndarray:
     return idx
 
 
-def score_select(q, proj, meta, G, M, scope="kv_head", head_softmax=False):
+def score_select(q, proj, meta, G, M, scope="kv_head", head_softmax=False, meta_exp=0):
     """O2..O6 chained.  Returns (idx [B,S,M'], R [B,S,NG]).  With head_softmax the per-head scores
     pass through `softmax_over_context` before the head sum (the other reading of "attention
-    scores" in Sec. 4.3)."""
+    scores" in Sec. 4.3).  `meta` holds the stored values of K_lr * 2^-meta_exp (meta_exp = 0 except
+    for 8-bit metadata): the scores are those of meta * 2^meta_exp."""
     Hkv = proj.shape[0]
+    if meta_exp:
+        meta = np.ldexp(np.asarray(meta, dtype=np.float64), int(meta_exp))
     s = head_scores(lowrank_query(q, proj), meta, Hkv)
     if head_softmax:
         s = softmax_over_context(s, q.shape[2], G)

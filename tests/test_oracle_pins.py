@@ -710,3 +710,111 @@ def test_head_softmax_changes_the_ranking_only_across_heads():
     want = [math.exp(4) / z0 + 1 / z1, 1 / z0 + math.exp(5) / z1, 1 / z0 + math.exp(4.875) / z1,
             1 / z0 + math.exp(4.875) / z1]
     assert np.allclose(R_soft[0, 0], want, atol=1e-14) and soft[0, 0, 0] == 0
+
+
+# ------------------------------------------------------------------------------------------
+# 8-bit metadata: the E4M3 storage format (reading of "precision can be traded", Sec. 4.1 / 4.2)
+# ------------------------------------------------------------------------------------------
+def _e4m3_golden():
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "e4m3_format.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                bits, val = line.split()
+                rows.append((int(bits.replace(".", ""), 2), float(val)))
+    return rows
+
+
+def test_e4m3_table_matches_the_published_format_and_torch():
+    table = O.e4m3_decode_table()
+    for code, val in _e4m3_golden():
+        if np.isnan(val):
+            assert np.isnan(table[code])
+        else:
+            assert table[code] == val and np.signbit(table[code]) == np.signbit(val), (code, val)
+    import torch
+    ref = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(np.isnan(table), np.isnan(ref))
+    ok = ~np.isnan(ref)
+    assert np.array_equal(table[ok], ref[ok])
+
+
+def _nearest_by_brute_force(x):
+    """Nearest finite table entry of the same sign; of two equally near the one with the even code."""
+    table = O.e4m3_decode_table()
+    best = None
+    for code in range(256):
+        v = table[code]
+        if np.isnan(v) or (code >= 128) != bool(np.signbit(x)):
+            continue
+        key = (abs(v - x), code & 1)
+        if best is None or key < best[0]:
+            best = (key, code)
+    return best[1]
+
+
+def test_e4m3_round_is_nearest_with_ties_to_even_and_saturates():
+    # hand-worked: halfway cases go to the even mantissa; beyond 448 everything saturates
+    cases = {1.0625: 1.0, 1.1875: 1.25, -1.0625: -1.0, 2.0 ** -10: 0.0, 3 * 2.0 ** -10: 2.0 ** -8,
+             460.0: 448.0, 464.0: 448.0, 1000.0: 448.0, -1e9: -448.0, 0.0: 0.0, 0.0146484375: 0.0146484375 + 2.0 ** -10,
+             15.5: 16.0, 0.99: 1.0, 447.9: 448.0, 2.0 ** -6 - 2.0 ** -10: 2.0 ** -6}
+    # (0.0146484375 = 7.5 * 2^-9 lies halfway between the largest subnormal 7 * 2^-9 and the smallest
+    # normal 8 * 2^-9: it goes to the even one, 8 * 2^-9 = 2^-6)
+    for x, want in cases.items():
+        v, code = O.e4m3_round(np.array([x]))
+        assert v[0] == want, (x, v[0], want)
+        assert O.e4m3_decode_table()[code[0]] == want
+    rng = np.random.default_rng(5)
+    xs = np.concatenate([rng.standard_normal(400) * s for s in (1e-3, 0.02, 1.0, 30.0, 300.0)])
+    xs = np.concatenate([xs, np.array([(k + 0.5) * 2.0 ** -9 for k in range(16)])])      # subnormal halfway points
+    v, code = O.e4m3_round(xs)
+    for x, c in zip(xs, code):
+        assert c == _nearest_by_brute_force(np.clip(x, -448, 448)), x
+    # an independent library conversion agrees wherever it is defined (it has no saturation)
+    import torch
+    inside = np.abs(xs) < 464
+    ref = torch.from_numpy(xs[inside]).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    nz = v[inside] != 0                                                              # the sign of a rounded zero is free
+    assert np.array_equal(code[inside][nz], ref[nz])
+
+
+def test_e4m3_planted_rounding_mistakes_are_caught(monkeypatch):
+    xs = np.array([1.0625, 1.1875, 3 * 2.0 ** -10, 0.99])
+    good = O.e4m3_round(xs)[0]
+    monkeypatch.setattr(np, "rint", lambda a: np.floor(a + 0.5))          # halves away from zero
+    assert not np.array_equal(O.e4m3_round(xs)[0], good)
+    monkeypatch.setattr(np, "rint", np.floor)                             # truncation
+    assert not np.array_equal(O.e4m3_round(xs)[0], good)
+
+
+def test_project_keys_e4m3_rounds_the_exact_product_once():
+    rng = np.random.default_rng(11)
+    B, Hkv, N, d, r = 1, 2, 6, 4, 4
+    K = (rng.integers(-8, 9, size=(B, Hkv, N, d)) / 4.0).astype(np.float32)       # dyadic: exact in every type
+    proj = (rng.integers(-8, 9, size=(Hkv, d, r)) / 8.0).astype(np.float32)
+    for meta_heads in (1, Hkv):
+        for e in (0, 2, -1):
+            meta = O.project_keys(K, proj, meta_heads, "e4m3", meta_exp=e)
+            table = O.e4m3_decode_table()
+            for m in range(meta_heads):
+                for n in range(N):
+                    for j in range(r):
+                        heads = range(Hkv) if meta_heads == 1 else [m]
+                        exact = sum(Fraction(float(K[0, g, n, c])) * Fraction(float(proj[g, c, j])) for g in heads for c in range(d))
+                        exact = float(exact / Fraction(2) ** e)
+                        assert meta[0, m, n, j] == table[_nearest_by_brute_force(exact)] or (meta[0, m, n, j] == 0 and table[_nearest_by_brute_force(exact)] == 0)
+
+
+def test_score_select_undoes_the_power_of_two_of_8bit_metadata():
+    """Scores of meta * 2^e stored as (meta, e) equal the scores of meta * 2^e passed directly; the
+    selection does not depend on e as long as nothing saturates."""
+    wl = W.CONFIGS[1].reduced("e4m3-sel", n_ctx=256, top_k=8)
+    li = W.make_layer(wl, 0, 1)
+    meta8 = O.project_keys(li.K, li.proj, 1, "e4m3", meta_exp=-2)
+    idx_a, R_a = O.score_select(li.q, li.proj, meta8, wl.group_size, wl.top_k, meta_exp=-2)
+    idx_b, R_b = O.score_select(li.q, li.proj, (meta8.astype(np.float64) * 0.25), wl.group_size, wl.top_k)
+    assert np.array_equal(idx_a, idx_b) and np.allclose(R_a, R_b, rtol=0, atol=0)
+    # and the 8-bit cache still ranks like the fp16 one on most groups (reported, not a pin of quality)
+    meta16 = O.project_keys(li.K, li.proj, 1, "f32")
+    idx_c, _ = O.score_select(li.q, li.proj, meta16, wl.group_size, wl.top_k)
+    assert len(set(idx_a[0, 0]) & set(idx_c[0, 0])) >= wl.top_k // 2
