@@ -76,7 +76,9 @@ typedef enum {
   KVSWAP_ERR_TIMEOUT = 10     /* a kernel gave up a bounded wait; its outputs are invalid     */
 } kvswap_status;
 
-typedef enum { KVSWAP_F32 = 0, KVSWAP_BF16 = 1, KVSWAP_F16 = 2 } kvswap_dtype;
+/* KVSWAP_E4M3 is a metadata type only: the 8-bit floating-point format E4M3 (1 sign, 4 exponent bits
+ * with bias 7, 3 mantissa bits; no infinities; S.1111.111 = NaN; largest finite value 448). */
+typedef enum { KVSWAP_F32 = 0, KVSWAP_BF16 = 1, KVSWAP_F16 = 2, KVSWAP_E4M3 = 3 } kvswap_dtype;
 typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_scope;
 
 /*
@@ -97,8 +99,18 @@ typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_sco
  *       lie in [0, heads per scope].  Two passes over the metadata (tensor cores for joint
  *       fp16 metadata with r = 32 and H_q <= 32, general fp32 kernels otherwise).
  *       KVSWAP_ERR_UNSUPPORTED if H_q * (r + 2) floats exceed 160 KB.
+ *   KVSWAP_META_EXP(e)     bits 8..15: a power of two for 8-bit metadata (meta_dtype = KVSWAP_E4M3),
+ *       -64 <= e <= 63, 0 for every other metadata type.  The paper leaves the precision of the
+ *       compact cache open ("can be flexibly traded", Sec. 4.1 / 4.2); with KVSWAP_E4M3 a row of
+ *       K_lr takes r bytes: kvswap_project_keys stores round(K_lr * 2^-e) -- one round-to-nearest-
+ *       even, magnitudes beyond 448 saturate -- and kvswap_score_select scores the stored values
+ *       times 2^e.  The ranking does not depend on e; choose it so that |K_lr| * 2^-e stays below
+ *       448 and the bulk of the values above 2^-6 (e = 0 suits keys of unit scale).  Supported for
+ *       r = 32, G a power of two <= 32 and dense metadata rows (else KVSWAP_ERR_UNSUPPORTED); not with
+ *       KVSWAP_SCORE_SOFTMAX.
  */
 enum { KVSWAP_INPUTS_SETTLED = 1, KVSWAP_SCORE_SOFTMAX = 2 };
+#define KVSWAP_META_EXP(e) ((int32_t)(((uint32_t)(e) & 0xffu) << 8))
 
 /*
  * Problem description shared by all calls.
@@ -107,7 +119,7 @@ enum { KVSWAP_INPUTS_SETTLED = 1, KVSWAP_SCORE_SOFTMAX = 2 };
  * A stride of 0 means "dense": the natural stride of the contiguous tensor.
  * Supported ranges: d in {64, 128}; r a multiple of 4 with 4 <= r <= 256; G >= 1; M >= 1;
  * rho >= 1; G <= 1024; M * G <= 2^30; kv_dtype in {F32, BF16, F16}; q_dtype = kv_dtype or F32; meta_dtype in
- * {F32, F16}.
+ * {F32, F16, E4M3}.
  */
 typedef struct {
   int32_t batch, n_ctx, n_q_heads, n_kv_heads, head_dim; /* B, N, H_q, H_kv, d            */

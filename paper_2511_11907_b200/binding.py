@@ -14,10 +14,15 @@ from typing import Optional
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libkvswap.so")
 
-KVSWAP_F32, KVSWAP_BF16, KVSWAP_F16 = 0, 1, 2
+KVSWAP_F32, KVSWAP_BF16, KVSWAP_F16, KVSWAP_E4M3 = 0, 1, 2, 3
 KVSWAP_SCOPE_KV_HEAD, KVSWAP_SCOPE_ALL_HEADS = 0, 1
 KVSWAP_INPUTS_SETTLED = 1      # kvswap_shape.flags
 KVSWAP_SCORE_SOFTMAX = 2
+
+
+def KVSWAP_META_EXP(e: int) -> int:
+    """kvswap_shape.flags bits of the power of two 8-bit metadata is stored with."""
+    return (int(e) & 0xff) << 8
 
 
 class KVSwapError(RuntimeError):

@@ -15,6 +15,7 @@ int dtype_bytes(int t) {
   switch (t) {
     case KVSWAP_F32: return 4;
     case KVSWAP_BF16: case KVSWAP_F16: return 2;
+    case KVSWAP_E4M3: return 1;
     default: return 0;
   }
 }
@@ -27,11 +28,14 @@ int resolve(const kvswap_shape* s, Problem* p) {
   if (s->n_q_heads % s->n_kv_heads != 0) return KVSWAP_ERR_SHAPE;
   if (s->meta_heads != 1 && s->meta_heads != s->n_kv_heads) return KVSWAP_ERR_SHAPE;
   if (s->scope != KVSWAP_SCOPE_KV_HEAD && s->scope != KVSWAP_SCOPE_ALL_HEADS) return KVSWAP_ERR_SHAPE;
-  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED | KVSWAP_SCORE_SOFTMAX)) != 0) return KVSWAP_ERR_SHAPE;
+  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED | KVSWAP_SCORE_SOFTMAX | 0xff00)) != 0) return KVSWAP_ERR_SHAPE;
+  const int meta_exp = int(int8_t((s->flags >> 8) & 0xff));
+  if (meta_exp < -64 || meta_exp > 63 || (meta_exp != 0 && s->meta_dtype != KVSWAP_E4M3)) return KVSWAP_ERR_SHAPE;
   if (s->n_ctx > (1 << 30) || s->batch > 65535 || s->n_q_heads > 4096) return KVSWAP_ERR_SHAPE;
   const int ekv = dtype_bytes(s->kv_dtype), em = dtype_bytes(s->meta_dtype), eq = dtype_bytes(s->q_dtype);
   if (ekv == 0 || em == 0 || eq == 0) return KVSWAP_ERR_DTYPE;
-  if (s->meta_dtype == KVSWAP_BF16) return KVSWAP_ERR_DTYPE;   // metadata is fp16 or fp32
+  if (s->meta_dtype == KVSWAP_BF16) return KVSWAP_ERR_DTYPE;   // metadata is fp32, fp16 or E4M3
+  if (s->kv_dtype == KVSWAP_E4M3 || s->q_dtype == KVSWAP_E4M3) return KVSWAP_ERR_DTYPE;   // a metadata type only
   if (s->q_dtype != KVSWAP_F32 && s->q_dtype != s->kv_dtype) return KVSWAP_ERR_DTYPE;  // q: fp32 or K/V's type
   if (s->head_dim != 64 && s->head_dim != 128) return KVSWAP_ERR_UNSUPPORTED;
   if (s->rank % 4 != 0 || s->rank > 256 || s->group_size > 1024) return KVSWAP_ERR_UNSUPPORTED;
@@ -42,7 +46,8 @@ int resolve(const kvswap_shape* s, Problem* p) {
   p->B = s->batch; p->N = s->n_ctx; p->Hq = s->n_q_heads; p->Hkv = s->n_kv_heads; p->d = s->head_dim;
   p->r = s->rank; p->Hm = s->meta_heads; p->G = s->group_size; p->M = s->top_k;
   p->kv_dtype = s->kv_dtype; p->meta_dtype = s->meta_dtype; p->q_dtype = s->q_dtype; p->scope = s->scope;
-  p->flags = s->flags;
+  p->flags = s->flags & 0xff;
+  p->meta_exp = meta_exp;
 
   p->kv_sn = s->kv_stride_n ? s->kv_stride_n : p->d;
   p->kv_sh = s->kv_stride_h ? s->kv_stride_h : int64_t(p->N) * p->kv_sn;
@@ -62,6 +67,9 @@ int resolve(const kvswap_shape* s, Problem* p) {
   p->Su = (p->Hm == 1) ? p->S : p->Hkv;
   p->score_pitch = p->NG;
   if ((p->flags & KVSWAP_SCORE_SOFTMAX) && !score_softmax_supported(*p)) return KVSWAP_ERR_UNSUPPORTED;
+  // 8-bit metadata is read by the streaming tensor-core scorer only
+  if (p->meta_dtype == KVSWAP_E4M3 && ((p->flags & KVSWAP_SCORE_SOFTMAX) || p->r != 32 || (p->NG > 0 && !score_stream_supported(*p))))
+    return KVSWAP_ERR_UNSUPPORTED;
   return KVSWAP_OK;
 }
 
@@ -73,7 +81,7 @@ static int workspace_score_pitch(const Problem& p) { return (std::max(p.NG, 1) +
 // batch and head counts alone, at a fixed place in front of everything else, so that one workspace
 // keeps them zero between calls while the context grows.
 static bool hist_capable(const Problem& p) {
-  return p.meta_dtype == KVSWAP_F16 && p.r == 32 && int64_t(p.B) * p.S <= 1024;
+  return (p.meta_dtype == KVSWAP_F16 || p.meta_dtype == KVSWAP_E4M3) && p.r == 32 && int64_t(p.B) * p.S <= 1024;
 }
 
 // The scorer counts the leading digit of every group score's key and the TopK starts from those

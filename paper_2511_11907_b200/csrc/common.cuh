@@ -18,7 +18,8 @@ constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs; grids are sized in multi
 struct Problem {
   int B, N, Hq, Hkv, d, r, Hm, G, M;
   int kv_dtype, meta_dtype, q_dtype, scope;
-  int flags;   // KVSWAP_INPUTS_SETTLED
+  int flags;   // KVSWAP_INPUTS_SETTLED, KVSWAP_SCORE_SOFTMAX
+  int meta_exp;   // 8-bit metadata stores K_lr * 2^-meta_exp (0 for the other types)
   int64_t kv_sb, kv_sh, kv_sn;
   int64_t meta_sb, meta_sh, meta_sn;
   int rho;   // H_q / H_kv
@@ -154,6 +155,22 @@ __device__ __forceinline__ void widen16B(const uint4& v, float (&f)[8], __half) 
     float2 t = __half22float2(h[i]);
     f[2 * i] = t.x; f[2 * i + 1] = t.y;
   }
+}
+
+// Storage of one E4M3 value (8-bit metadata): 1 sign, 4 exponent bits with bias 7, 3 mantissa bits.
+struct e4m3_t { uint8_t bits; };
+
+// Two fp32 values -> two E4M3 bytes (lo in the low byte): round to nearest even, magnitudes beyond
+// 448 saturate.
+__device__ __forceinline__ uint16_t to_e4m3x2(float lo, float hi) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// 2^-meta_exp, the factor 8-bit metadata is stored with (1 for the other types).
+__device__ __forceinline__ float meta_store_scale(const Problem& p) {
+  return __uint_as_float(uint32_t(127 - p.meta_exp) << 23);
 }
 
 // 16-byte read-only global load that does not allocate in L1 (streamed once).

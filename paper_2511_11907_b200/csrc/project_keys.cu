@@ -104,7 +104,9 @@ project_keys_kernel(Problem p, const ProjectTable tab, int tiles, int n_begin, i
     for (int j = 0; j < RC; ++j) {
       const int col = lane + 32 * j;
       if (col < p.r) {
-        if constexpr (sizeof(META_T) == 2) Mo[int64_t(n) * p.meta_sn + col] = __float2half_rn(acc[i][j]);
+        if constexpr (sizeof(META_T) == 1)
+          Mo[int64_t(n) * p.meta_sn + col].bits = uint8_t(to_e4m3x2(acc[i][j] * meta_store_scale(p), 0.f) & 0xffu);
+        else if constexpr (sizeof(META_T) == 2) Mo[int64_t(n) * p.meta_sn + col] = __float2half_rn(acc[i][j]);
         else Mo[int64_t(n) * p.meta_sn + col] = acc[i][j];
       }
     }
@@ -354,7 +356,9 @@ project_group_kernel(Problem p, const ProjectTable tab, int n_begin, int n_token
 #pragma unroll
     for (int k = 0; k < 8; ++k) s += part_sum[k][col];
     META_T* out = meta + int64_t(b) * p.meta_sb + int64_t(head_out) * p.meta_sh + int64_t(n) * p.meta_sn + col;
-    if constexpr (sizeof(META_T) == 2) *out = __float2half_rn(s); else *out = s;
+    if constexpr (sizeof(META_T) == 1) out->bits = uint8_t(to_e4m3x2(s * meta_store_scale(p), 0.f) & 0xffu);
+    else if constexpr (sizeof(META_T) == 2) *out = __float2half_rn(s);
+    else *out = s;
   }
 }
 
@@ -380,6 +384,7 @@ template <typename KV_T>
 cudaError_t dispatch_rc_meta(const Problem& p, const ProjectTable& tab, int n_layers, int n_begin, int n_end,
                              cudaStream_t st) {
   if (p.meta_dtype == KVSWAP_F16) return dispatch_rc<KV_T, __half>(p, tab, n_layers, n_begin, n_end, st);
+  if (p.meta_dtype == KVSWAP_E4M3) return dispatch_rc<KV_T, e4m3_t>(p, tab, n_layers, n_begin, n_end, st);
   return dispatch_rc<KV_T, float>(p, tab, n_layers, n_begin, n_end, st);
 }
 
@@ -398,7 +403,7 @@ template <typename KV_T>
 cudaError_t dispatch_meta(const Problem& p, const void* K, const float* proj, void* meta, int n_begin, int n_end,
                           bool tensor_cores, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
-  if (tensor_cores) {
+  if (tensor_cores && p.meta_dtype != KVSWAP_E4M3) {      // (8-bit metadata: tcgen05 path or the fp32 kernel)
     if (p.meta_dtype == KVSWAP_F16) {
       if (try_launch_mma<__half>(p, K, proj, meta, n_begin, n_end, st, &e)) return e;
     } else if (try_launch_mma<float>(p, K, proj, meta, n_begin, n_end, st, &e)) {

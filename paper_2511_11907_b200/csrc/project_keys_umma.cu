@@ -195,7 +195,17 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
         const int n = n_begin + tile * kTileM + row;
         if (n < n_end) {
           META_T* dst = meta + int64_t(b) * p.meta_sb + int64_t(hm) * p.meta_sh + int64_t(n) * p.meta_sn;
-          if constexpr (sizeof(META_T) == 2) {
+          if constexpr (sizeof(META_T) == 1) {             // E4M3: the row is kR bytes
+            const float sc = meta_store_scale(p);
+            uint32_t w[kR / 4];
+#pragma unroll
+            for (int j = 0; j < kR / 4; ++j)
+              w[j] = uint32_t(to_e4m3x2(acc[4 * j] * sc, acc[4 * j + 1] * sc)) |
+                     (uint32_t(to_e4m3x2(acc[4 * j + 2] * sc, acc[4 * j + 3] * sc)) << 16);
+#pragma unroll
+            for (int j = 0; j < kR / 16; ++j)
+              reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+          } else if constexpr (sizeof(META_T) == 2) {
             uint32_t w[kR / 2];
 #pragma unroll
             for (int j = 0; j < kR / 2; ++j) {
@@ -270,7 +280,8 @@ bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* 
     kern<<<ctas, kThreadsUmma, smem, st>>>(p, map_k, map_b, meta_t, n_begin, n_end, tiles_per_row, err);
     return cudaGetLastError();
   };
-  if (p.meta_dtype == KVSWAP_F16) *result = go(project_keys_umma_kernel<__half>, static_cast<__half*>(meta));
+  if (p.meta_dtype == KVSWAP_E4M3) *result = go(project_keys_umma_kernel<e4m3_t>, static_cast<e4m3_t*>(meta));
+  else if (p.meta_dtype == KVSWAP_F16) *result = go(project_keys_umma_kernel<__half>, static_cast<__half*>(meta));
   else *result = go(project_keys_umma_kernel<float>, static_cast<float*>(meta));
   return true;
 }

@@ -36,6 +36,8 @@
 // global histograms are zero on entry and left zero by the TopK kernel that starts from them
 // (topk_select.cu; kvswap_workspace_init clears them once).
 #include <algorithm>
+#include <cmath>
+#include <type_traits>
 
 #include "async_copy.cuh"
 #include "common.cuh"
@@ -45,16 +47,18 @@ namespace kvswap {
 namespace {
 
 constexpr uint32_t kFull = 0xffffffffu;
-constexpr int kTileRows = 32;
-constexpr int kRowBytes = 64;
-constexpr int kTileBytes = kTileRows * kRowBytes;
+constexpr int kTileBytes = 2048;                          // one stage: 32 fp16 rows of 64 bytes, or 64 E4M3 rows of 32 bytes
+template <bool FP8> struct Tile {
+  static constexpr int kRowBytes = FP8 ? 32 : 64;
+  static constexpr int kRows = kTileBytes / kRowBytes;
+};
 constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kDepth = 4;
 constexpr int kCols = 8;                                  // scores per metadata row and instruction
 constexpr int kHistWords = kCols * kKeyTopBins / 2;       // two 16-bit counters per word
 constexpr int kMaxSets = 4;                               // row sets one CTA may touch when it builds the queries itself
-constexpr int kMaxTilesPerWarp = 65535 / kTileRows;       // bound that keeps a 16-bit counter from overflowing (G = 1)
+constexpr int kMaxTilesPerCta = 65535 / 64;                // bound that keeps a 16-bit counter from overflowing (64 rows, G = 1)
 
 struct Smem {
   unsigned char tiles[kWarps * kDepth * kTileBytes];      // 128 KB of stages
@@ -69,12 +73,13 @@ struct StreamArgs {
   const void* q;            // fused: [B, H_q, d] q_dtype
   const float* proj;        // fused: [H_kv, d, r]
   const float* uq;          // not fused: [B, Su, r] from the low-rank query kernel
-  const __half* meta;
+  const unsigned char* meta;
   float* scores;
   uint32_t* top_hist;       // NULL, or [B * S, 4096] 16-bit counters, two per word
   int tiles_per_row, n_sub, n_rests;
   int vset_items, ctas_per_vset;   // work split: virtual sets of vset_items items, each shared by ctas_per_vset CTAs
   int base, rem;            // tiles per warp within a virtual set: base, +1 for the first rem warps
+  float meta_scale;         // 2^meta_exp (1 unless the metadata is 8-bit)
   uint32_t* err;
 };
 
@@ -178,10 +183,14 @@ __device__ void build_queries(const Problem& p, const void* q, const float* __re
   }
 }
 
-template <int GS, bool FUSED>                        // GS = log2(G), 0..5
+// FP8: the metadata is E4M3 (rows of 32 bytes, 64 per tile); every value converts to fp16 exactly, so
+// the product below is the same with twice the rows per byte.
+template <int GS, bool FUSED, bool FP8>              // GS = log2(G), 0..5
 __global__ void __launch_bounds__(kThreads, 1)
 score_stream_kernel(Problem p, StreamArgs a) {
   constexpr int g_shift = GS;
+  constexpr int kTileRows = Tile<FP8>::kRows;
+  constexpr int kRowBytes = Tile<FP8>::kRowBytes;
   extern __shared__ __align__(128) unsigned char dyn[];
   Smem* sm = reinterpret_cast<Smem*>(dyn);
 
@@ -213,19 +222,19 @@ score_stream_kernel(Problem p, StreamArgs a) {
   int c_tile = f_tile, c_rest = f_rest;                                           // next item to consume
 
   const uint32_t ring = smem_addr(sm->tiles) + uint32_t(warp) * kDepth * kTileBytes;
-  const __half* f_base = nullptr;                   // metadata of the fill cursor's (sequence, head)
+  const unsigned char* f_base = nullptr;            // metadata of the fill cursor's (sequence, head)
   int f_base_rest = -1;
   auto fill = [&](int stage) {
     if (lane == 0) {
       if (f_rest != f_base_rest) {                  // divisions only when the cursor enters a new row set
         f_base_rest = f_rest;
         const int bh = f_rest / a.n_sub;
-        f_base = a.meta + int64_t(bh / hm_count) * p.meta_sb + int64_t(bh % hm_count) * p.meta_sh;
+        f_base = a.meta + (int64_t(bh / hm_count) * p.meta_sb + int64_t(bh % hm_count) * p.meta_sh) * (FP8 ? 1 : 2);
       }
       const int rows = min(kTileRows, rows_total - f_tile * kTileRows);
       const uint32_t bar = smem_addr(&sm->full[warp * kDepth + stage]);
       mbar_arrive_expect_tx(bar, uint32_t(rows) * kRowBytes);
-      bulk_g2s(ring + uint32_t(stage) * kTileBytes, f_base + int64_t(f_tile) * kTileRows * p.meta_sn,
+      bulk_g2s(ring + uint32_t(stage) * kTileBytes, f_base + int64_t(f_tile) * kTileRows * kRowBytes,
                uint32_t(rows) * kRowBytes, bar);
     }
     if (++f_tile == a.tiles_per_row) { f_tile = 0; ++f_rest; }
@@ -303,7 +312,7 @@ score_stream_kernel(Problem p, StreamArgs a) {
       int sh = 0;
       if (mx > 0.f && mx < INFINITY) sh = min(120, max(-113, 14 - (int((__float_as_uint(mx) >> 23) & 0xffu) - 127)));
       const float scale = __uint_as_float(uint32_t(sh + 127) << 23);
-      inv = __uint_as_float(uint32_t(127 - sh) << 23);
+      inv = __uint_as_float(uint32_t(127 - sh) << 23) * a.meta_scale;     // also undoes the 8-bit cache's power of two
       __half hi[8], lo[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -331,15 +340,25 @@ score_stream_kernel(Problem p, StreamArgs a) {
     if (!__all_sync(kFull, mbar_wait(smem_addr(&sm->full[warp * kDepth + stage]), phase))) { timed_out = true; break; }
     const int rows = min(kTileRows, rows_total - tile * kTileRows);   // a multiple of G: groups never straddle tiles
     const int ngt = rows >> g_shift;                // groups in this tile
-    const uint32_t base = ring + uint32_t(stage) * kTileBytes + uint32_t(lane) * 16u;
+    const uint32_t base = ring + uint32_t(stage) * kTileBytes + uint32_t(lane) * (kRowBytes / 4);
     float* dst = my_row + ((tile * kTileRows) >> g_shift);           // first group of the tile in this lane's row
-    float mine = 0.f;                               // G = 8: the group of read `qt` is this lane's to publish
+    float mine[kTileRows / 32] = {};                // G = 8: the groups of reads qt, qt + 4, .. are this lane's to publish
 #pragma unroll
     for (int it = 0; it < kTileRows / 8; ++it) {
       if (it * 8 < rows) {
-        uint32_t w[4];
-        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
-                     : "r"(base + uint32_t(it) * 8u * kRowBytes));
+        uint32_t w[4];                              // entries 8t .. 8t+7 of row g as fp16 pairs
+        if constexpr (FP8) {
+          uint32_t b8[2];
+          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(b8[0]), "=r"(b8[1]) : "r"(base + uint32_t(it) * 8u * kRowBytes));
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint16_t pair = uint16_t(b8[i >> 1] >> ((i & 1) * 16));
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(w[i]) : "h"(pair));
+          }
+        } else {
+          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
+                       : "r"(base + uint32_t(it) * 8u * kRowBytes));
+        }
         float d[4] = {0.f, 0.f, 0.f, 0.f};          // d[0], d[1]: head products of tokens 2t, 2t+1; d[2], d[3]: remainder products
 #pragma unroll
         for (int j = 0; j < 2; ++j) mma16816(d, ahl[j][0], alh[j][0], ahl[j][1], alh[j][1], w[2 * j], w[2 * j + 1]);
@@ -356,12 +375,12 @@ score_stream_kernel(Problem p, StreamArgs a) {
           else if constexpr (GS == 2) {
             if (scope_ok && (qt & 1) == 0 && it * 2 + (qt >> 1) < ngt) publish(dst + it * 2 + (qt >> 1), m * inv);
           }
-          else if constexpr (GS == 3) { if (qt == it) mine = m; }
+          else if constexpr (GS == 3) { if (qt == (it & 3)) mine[it >> 2] = m; }
           else {                                                 // G = 16 or 32: 2 or 4 reads per group
             run = fmaxf(run, m);
             if (((it + 1) & ((1 << (GS - 3)) - 1)) == 0) {
               const int gi = it >> (GS - 3);
-              if (scope_ok && qt == gi) publish(dst + gi, run * inv);
+              if (scope_ok && qt == (gi & 3)) publish(dst + gi, run * inv);
               run = -INFINITY;
             }
           }
@@ -369,7 +388,9 @@ score_stream_kernel(Problem p, StreamArgs a) {
       }
     }
     if constexpr (GS == 3) {
-      if (scope_ok && qt * 8 < rows) publish(dst + qt, mine * inv);
+#pragma unroll
+      for (int h = 0; h < kTileRows / 32; ++h)
+        if (scope_ok && (4 * h + qt) * 8 < rows) publish(dst + 4 * h + qt, mine[h] * inv);
     }
     __syncwarp();                                   // every lane has read the stage
     if (k + kDepth < my_tiles) fill(stage);
@@ -411,21 +432,25 @@ struct Plan {
   int ctas, vset_items, ctas_per_vset, base, rem;
   bool fused;
   bool counts;
+  bool fp8;
 };
 
 // Launch geometry of the streaming scorer for `p`; false when the shape does not take it.
 bool plan(const Problem& p, Plan* pl) {
-  if (p.meta_dtype != KVSWAP_F16 || p.NG < 1) return false;
+  const bool fp8 = p.meta_dtype == KVSWAP_E4M3;
+  if ((p.meta_dtype != KVSWAP_F16 && !fp8) || p.NG < 1) return false;
   int g_shift = -1;
   for (int s = 0; s <= 5; ++s) if ((1 << s) == p.G) g_shift = s;
   const bool one_term = (p.Hm == 1) || (p.scope == KVSWAP_SCOPE_KV_HEAD);
-  if (!one_term || g_shift < 0 || p.r * 2 != kRowBytes || p.meta_sn != p.r) return false;
+  const int row_bytes = fp8 ? 32 : 64, tile_rows = kTileBytes / row_bytes;
+  if (!one_term || g_shift < 0 || p.r * (fp8 ? 1 : 2) != row_bytes || p.meta_sn != p.r) return false;
   const int64_t rows_total = int64_t(p.NG) * p.G;
-  const int64_t tiles_per_row = (rows_total + kTileRows - 1) / kTileRows;
+  const int64_t tiles_per_row = (rows_total + tile_rows - 1) / tile_rows;
   const int n_sub = (p.Hm == 1) ? (p.S + kCols - 1) / kCols : 1;
   const int64_t n_rests = int64_t(p.B) * ((p.Hm == 1) ? 1 : p.Hkv) * n_sub;
   const int64_t items = n_rests * tiles_per_row;
   if (items >= (int64_t(1) << 30)) return false;
+  pl->fp8 = fp8;
   pl->g_shift = g_shift;
   pl->tiles_per_row = int(tiles_per_row); pl->n_sub = n_sub; pl->n_rests = int(n_rests);
   // One CTA per SM.  When the row sets divide the SMs (almost) evenly every row set gets its own CTAs,
@@ -448,7 +473,7 @@ bool plan(const Problem& p, Plan* pl) {
   const int64_t cta_items = int64_t(pl->base + 1) * kWarps;
   const int64_t sets_touched = (cta_items + tiles_per_row - 1) / tiles_per_row + 1;
   pl->fused = p.r == 32 && (p.d == 32 || p.d == 64 || p.d == 128) && sets_touched <= kMaxSets;
-  pl->counts = pl->base + 1 <= kMaxTilesPerWarp / kWarps;     // a CTA's counts stay below 2^16 per counter
+  pl->counts = (pl->base + 1) * kWarps <= kMaxTilesPerCta;   // a CTA's counts stay below 2^16 per counter
   return true;
 }
 
@@ -465,10 +490,11 @@ cudaError_t launch_score_stream(const Problem& p, const void* q, const float* pr
   if (top_hist != nullptr && !pl.counts) return cudaErrorInvalidValue;
   if (pl.fused ? (q == nullptr || proj == nullptr) : (uq == nullptr)) return cudaErrorInvalidValue;
   StreamArgs a;
-  a.q = q; a.proj = proj; a.uq = uq; a.meta = static_cast<const __half*>(meta); a.scores = scores;
+  a.q = q; a.proj = proj; a.uq = uq; a.meta = static_cast<const unsigned char*>(meta); a.scores = scores;
   a.top_hist = top_hist;
   a.tiles_per_row = pl.tiles_per_row; a.n_sub = pl.n_sub; a.n_rests = pl.n_rests;
   a.vset_items = pl.vset_items; a.ctas_per_vset = pl.ctas_per_vset; a.base = pl.base; a.rem = pl.rem;
+  a.meta_scale = exp2f(float(p.meta_exp));
   a.err = err;
   const size_t smem = sizeof(Smem) + 128;
   auto go = [&](auto kern) -> cudaError_t {
@@ -476,24 +502,21 @@ cudaError_t launch_score_stream(const Problem& p, const void* q, const float* pr
     if (e != cudaSuccess) return e;
     return launch_pdl(kern, dim3(pl.ctas), dim3(kThreads), smem, st, p, a);
   };
-  if (pl.fused) {
+  auto go_gs = [&](auto fused, auto fp8) -> cudaError_t {
+    constexpr bool F = decltype(fused)::value, E = decltype(fp8)::value;
     switch (pl.g_shift) {
-      case 0: return go(score_stream_kernel<0, true>);
-      case 1: return go(score_stream_kernel<1, true>);
-      case 2: return go(score_stream_kernel<2, true>);
-      case 3: return go(score_stream_kernel<3, true>);
-      case 4: return go(score_stream_kernel<4, true>);
-      default: return go(score_stream_kernel<5, true>);
+      case 0: return go(score_stream_kernel<0, F, E>);
+      case 1: return go(score_stream_kernel<1, F, E>);
+      case 2: return go(score_stream_kernel<2, F, E>);
+      case 3: return go(score_stream_kernel<3, F, E>);
+      case 4: return go(score_stream_kernel<4, F, E>);
+      default: return go(score_stream_kernel<5, F, E>);
     }
-  }
-  switch (pl.g_shift) {
-    case 0: return go(score_stream_kernel<0, false>);
-    case 1: return go(score_stream_kernel<1, false>);
-    case 2: return go(score_stream_kernel<2, false>);
-    case 3: return go(score_stream_kernel<3, false>);
-    case 4: return go(score_stream_kernel<4, false>);
-    default: return go(score_stream_kernel<5, false>);
-  }
+  };
+  using T = std::true_type;
+  using N = std::false_type;
+  if (pl.fused) return pl.fp8 ? go_gs(T(), T()) : go_gs(T(), N());
+  return pl.fp8 ? go_gs(N(), T()) : go_gs(N(), N());
 }
 
 }  // namespace kvswap

@@ -19,7 +19,7 @@ from . import binding as kv
 from . import runtime as rt
 from . import workloads as W
 
-_TD = {W.F32: torch.float32, W.BF16: torch.bfloat16, W.F16: torch.float16}
+_TD = {W.F32: torch.float32, W.BF16: torch.bfloat16, W.F16: torch.float16, W.E4M3: torch.float8_e4m3fn}
 
 
 def _gen(seed: int, salt: int, device) -> torch.Generator:

@@ -8,7 +8,7 @@ import torch
 from . import binding as kv
 from . import workloads as W
 
-_TORCH_DTYPE = {W.F32: torch.float32, W.BF16: torch.bfloat16, W.F16: torch.float16}
+_TORCH_DTYPE = {W.F32: torch.float32, W.BF16: torch.bfloat16, W.F16: torch.float16, W.E4M3: torch.float8_e4m3fn}
 
 
 def shape_for(wl: W.Workload, meta_heads: int = 1, scope: int = W.SCOPE_KV_HEAD, **override) -> kv.kvswap_shape:

@@ -32,6 +32,7 @@ BASE_SEED = 20251111
 
 # dtype tags (same integer values as the C enum kvswap_dtype)
 F32, BF16, F16 = 0, 1, 2
+E4M3 = 3          # 8-bit metadata only
 # scope tags (same integer values as the C enum kvswap_scope)
 SCOPE_KV_HEAD, SCOPE_ALL_HEADS = 0, 1
 

@@ -191,6 +191,22 @@ def test_tiered_step_validates_before_touching_the_gpu(lib):
     assert app(roomy, ctypes.byref(short_tables)) == 2                     # the grown context outruns the tables
 
 
+def test_8bit_metadata_shapes_are_validated(lib):
+    ok = good_shape(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.E4M3, rank=32, head_dim=128, group_size=8)
+    assert kv.kvswap_validate_shape(ok) == 0
+    assert kv.kvswap_validate_shape(ok.with_flags(kv.KVSWAP_META_EXP(-3))) == 0
+    assert kv.kvswap_workspace_bytes(ok) > 0
+    bad_rank = good_shape(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.E4M3, rank=16, head_dim=128, group_size=8)
+    assert kv.kvswap_validate_shape(bad_rank) == 6                     # the 8-bit rows are read by one scorer only
+    odd_group = good_shape(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.E4M3, rank=32, head_dim=128, group_size=3)
+    assert kv.kvswap_validate_shape(odd_group) == 6
+    assert kv.kvswap_validate_shape(ok.with_flags(kv.KVSWAP_SCORE_SOFTMAX)) == 6
+    assert kv.kvswap_validate_shape(good_shape().with_flags(kv.KVSWAP_META_EXP(2))) == 2     # an exponent without 8-bit metadata
+    assert kv.kvswap_validate_shape(good_shape(kv_dtype=W.E4M3)) == 3
+    assert kv.kvswap_validate_shape(good_shape(q_dtype=W.E4M3)) == 3
+    assert kv.kvswap_validate_shape(ok.with_flags(1 << 16)) == 2           # unknown flag bit
+
+
 def test_status_strings_and_version(lib):
     seen = {kv.status_string(i) for i in range(11)}
     assert len(seen) == 11 and "ok" in seen

@@ -51,23 +51,30 @@ def _grow_and_check(wl, n0, meta_heads, scope, check_at):
     S = shape_at(Nf).n_scopes
     scores = torch.empty((B, S, Nf // G), dtype=torch.float32, device="cuda")
 
-    meta_or = O.project_keys(li.K, li.proj, meta_heads, META_NAME[wl.meta_dtype])
-    tol = project_tolerance(li.K, li.proj, meta_heads, meta_or, wl.meta_dtype)
+    # The oracle's append (O8) is stepped beside the device, token by token, from the same start.
+    K_o, V_o = li.K[:, :, :n0].copy(), li.V[:, :, :n0].copy()
+    meta_o = O.project_keys(K_o[:, :, :n0 // G * G], li.proj, meta_heads, META_NAME[wl.meta_dtype])
+    tol = project_tolerance(li.K, li.proj, meta_heads, O.project_keys(li.K, li.proj, meta_heads, META_NAME[wl.meta_dtype]),
+                            wl.meta_dtype)
     for n in range(n0, Nf):
         flushed = kv.kvswap_append_kv(shape_at(n), K_all[:, :, n].contiguous(), V_all[:, :, n].contiguous(), K, V,
                                       proj, meta)
-        assert flushed == ((n + 1) % G == 0)
+        K_o, V_o, meta_o, flushed_o = O.append_kv(K_o, V_o, meta_o, li.K[:, :, n], li.V[:, :, n], li.proj, G,
+                                                  META_NAME[wl.meta_dtype])
+        assert flushed == flushed_o
         n1 = n + 1
         if n1 not in check_at:
             continue
         torch.cuda.synchronize()
-        # ---- the store and the compact cache ------------------------------------------------------
-        assert torch.equal(K[:, :, :n1], K_all[:, :, :n1]) and torch.equal(V[:, :, :n1], V_all[:, :, :n1])
+        # ---- the store and the compact cache against the oracle's ---------------------------------------
+        assert K_o.shape[2] == n1 and meta_o.shape[2] == n1 // G * G
+        assert np.array_equal(rt.to_host_f32(K[:, :, :n1]), K_o.astype(np.float32))
+        assert np.array_equal(rt.to_host_f32(V[:, :, :n1]), V_o.astype(np.float32))
         assert torch.isnan(K[:, :, n1:].float()).all() and torch.isnan(V[:, :, n1:].float()).all()   # nothing beyond
         ng = n1 // G
         meta_gpu = rt.to_host_f32(meta)
         assert np.all(np.isfinite(meta_gpu[:, :, :ng * G]))
-        err = np.abs(meta_gpu[:, :, :ng * G].astype(np.float64) - meta_or[:, :, :ng * G].astype(np.float64))
+        err = np.abs(meta_gpu[:, :, :ng * G].astype(np.float64) - meta_o.astype(np.float64))
         assert np.all(err <= tol[:, :, :ng * G]), f"compact cache error {err.max():.3e}"
         assert np.isnan(meta_gpu[:, :, ng * G:]).all()                  # rows of the open group are not built
         # ---- predictor and attention over the grown context ------------------------------------------
