@@ -533,6 +533,7 @@ def run_ours(args, wl):
     soft_us, _ = graph_call_us(torch, [(lambda l=l: kv.kvswap_score_select(shape_soft, q0[l], dw.proj[l], dw.meta[l], idx[l],
                                                                           nsel[l], None, ws)) for l in range(L)], 400)
     _, select_bytes = workload_bytes(wl, meta_heads, S)
+    fp8 = fp8_metadata_leg(torch, kv, rt, wl, dw, meta_heads, scope, idx, nsel, dev, peak) if wl.meta_dtype == W.F16 and wl.rank == 32 else None
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         cpu = cpu_baseline(wl, dw, meta_heads, args.scope, rt)
@@ -578,6 +579,7 @@ def run_ours(args, wl):
         "predictor_softmax_variant": {"kernel": "kvswap_score_select with KVSWAP_SCORE_SOFTMAX", "avg_ms": soft_us / 1e3,
                                       "frac": select_bytes / soft_us / 1e3 / peak,
                                       "algorithmic_bytes_per_launch": select_bytes},
+        "metadata_8bit": fp8,
         "prefill": {"project_keys_ms_all_layers": prefill_ms,
                     "keys_projected_per_sec": keys_per_step / prefill_ms * 1e3,
                     "read_gbs": L * wl.batch * wl.n_kv_heads * wl.n_ctx * wl.head_dim * esz[wl.kv_dtype] / prefill_ms / 1e6},
@@ -589,6 +591,38 @@ def run_ours(args, wl):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def fp8_metadata_leg(torch, kv, rt, wl, dw, meta_heads, scope, idx, nsel, dev, peak):
+    """The predictor over an 8-bit compact cache (KVSWAP_E4M3: half the bytes of the fp16 one): the
+    metadata of every layer rebuilt in that format, kvswap_score_select timed like the fp16 calls, and
+    how many of the fp16 predictor's groups it still selects (reported, not graded)."""
+    L, S = wl.layers, 1 if scope == W.SCOPE_ALL_HEADS else wl.n_kv_heads
+    wl8 = wl.reduced(wl.name + "-e4m3", meta_dtype=W.E4M3)
+    shape8 = rt.shape_for(wl8, meta_heads, scope)
+    ws8 = rt.alloc_workspace(shape8, dev)
+    meta8 = [torch.empty((wl.batch, meta_heads, wl.n_ctx, wl.rank), dtype=torch.uint8, device=dev) for _ in range(L)]
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    kv.kvswap_project_keys(shape8, dw.K[0], dw.proj[0], meta8[0], 0, wl.n_ctx, ws8)
+    torch.cuda.synchronize()
+    a.record()
+    for l in range(L):
+        kv.kvswap_project_keys(shape8, dw.K[l], dw.proj[l], meta8[l], 0, wl.n_ctx, ws8)
+    b.record()
+    torch.cuda.synchronize()
+    prefill_ms = a.elapsed_time(b)
+    q0 = dw.q_walk[0]
+    idx8, nsel8 = torch.empty_like(idx), torch.empty_like(nsel)
+    fns = [(lambda l=l: kv.kvswap_score_select(shape8, q0[l], dw.proj[l], meta8[l], idx8[l], nsel8[l], None, ws8)) for l in range(L)]
+    us, calls = graph_call_us(torch, fns)
+    torch.cuda.synchronize()
+    both = (idx8.unsqueeze(-1) == idx.unsqueeze(-2)).any(dim=-1) & (idx8 >= 0)
+    agree = float(both.float().sum() / (idx8 >= 0).float().sum())
+    nbytes = wl.batch * meta_heads * wl.n_ctx * wl.rank + 2 * wl.batch * S * wl.n_groups * 4 + wl.batch * S * wl.top_k * 4
+    return {"format": "E4M3, one byte per entry, power-of-two exponent 0", "avg_ms": us / 1e3, "launches_timed": calls,
+            "algorithmic_bytes_per_launch": nbytes, "achieved": nbytes / us / 1e3, "unit": "GB/s",
+            "frac": nbytes / us / 1e3 / peak, "prefill_ms_all_layers": prefill_ms,
+            "groups_shared_with_the_fp16_predictor": agree}
 
 
 def secondary_workloads(torch, kv, rt, DW, wl5, dw5, scope, idx, nsel, out, dev, peak, peak_kind):
