@@ -66,8 +66,6 @@ int resolve(const kvswap_shape* s, Problem* p) {
   p->Mp = std::min(p->M, p->NG);
   p->Su = (p->Hm == 1) ? p->S : p->Hkv;
   p->score_pitch = p->NG;
-  p->scorer_ctas = 0;
-  p->attn_slots = 0;
   if ((p->flags & KVSWAP_SCORE_SOFTMAX) && !score_softmax_supported(*p)) return KVSWAP_ERR_UNSUPPORTED;
   // 8-bit metadata is read by the streaming tensor-core scorer only
   if (p->meta_dtype == KVSWAP_E4M3 && ((p->flags & KVSWAP_SCORE_SOFTMAX) || p->r != 32 || (p->NG > 0 && !score_stream_supported(*p))))

@@ -27,9 +27,6 @@ struct Problem {
   int NG;    // complete groups
   int Mp;    // min(M, NG)
   int Su;    // rows of the low-rank query buffer per sequence (see score_pool.cu)
-  // Set by kvswap_decode_step when the predictor and the attention share the GPU (0 = each has it alone):
-  int scorer_ctas;   // CTAs of half an SM the streaming scorer may use
-  int attn_slots;    // CTA slots (two per SM) the split-K gather plans for
   int score_pitch;   // floats between rows of the group-score buffer: NG in a caller's buffer, padded in the workspace
 };
 

@@ -52,19 +52,18 @@ template <bool FP8> struct Tile {
   static constexpr int kRowBytes = FP8 ? 32 : 64;
   static constexpr int kRows = kTileBytes / kRowBytes;
 };
-constexpr int kWarpsFull = 16;                            // one CTA per SM: the whole GPU scores
-constexpr int kWarpsLight = 8;                            // half an SM per CTA: the scorer shares the GPU with the attention
+constexpr int kWarps = 16;
+constexpr int kThreads = kWarps * 32;
 constexpr int kDepth = 4;
 constexpr int kCols = 8;                                  // scores per metadata row and instruction
 constexpr int kHistWords = kCols * kKeyTopBins / 2;       // two 16-bit counters per word
 constexpr int kMaxSets = 4;                               // row sets one CTA may touch when it builds the queries itself
 constexpr int kMaxTilesPerCta = 65535 / 64;                // bound that keeps a 16-bit counter from overflowing (64 rows, G = 1)
 
-template <int WARPS, bool HIST>
-struct SmemT {
-  unsigned char tiles[WARPS * kDepth * kTileBytes];       // 128 KB (64 KB) of stages
-  uint32_t hist[HIST ? kHistWords : 4];                   // 64 KB; the light scorer counts in global memory
-  unsigned long long full[WARPS * kDepth];
+struct Smem {
+  unsigned char tiles[kWarps * kDepth * kTileBytes];      // 128 KB of stages
+  uint32_t hist[kHistWords];                              // 64 KB
+  unsigned long long full[kWarps * kDepth];
   float qsum[8 * 128];                                    // summed queries of up to 8 KV heads
   float upart[32 * 32];                                   // partial products, [item][column]
   float urow[kMaxSets][kCols * 32];                       // summed low-rank queries per row set of the CTA
@@ -116,10 +115,8 @@ __device__ __forceinline__ RowSet row_set(const Problem& p, int rest, int n_sub)
 // it requests the adapter rows of its (at most two) items first, then the CTA sums the query
 // heads into shared memory, so that both loads share one round trip.  The partial products are
 // added in a fixed order.  All threads call.
-template <int WARPS, typename SM>
 __device__ void build_queries(const Problem& p, const void* q, const float* __restrict__ proj, RowSet rs,
-                              SM* sm, float* urow) {
-  constexpr int kThreads = WARPS * 32;
+                              Smem* sm, float* urow) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool joint = p.Hm == 1;
   const bool all_heads = joint && p.scope == KVSWAP_SCOPE_ALL_HEADS;
@@ -132,27 +129,17 @@ __device__ void build_queries(const Problem& p, const void* q, const float* __re
   const int d_shift = ch_shift + 5;
   for (int t0 = 0; t0 < n_terms; t0 += 8) {
     const int nt = min(8, n_terms - t0);
-    const int n_items = nt << ch_shift;                            // <= 32
-    // A warp takes items two at a time (warp, warp + WARPS; then + 2 WARPS, ...).  The adapter rows
-    // of its first pair are requested before the query heads are summed, so both loads share a round trip.
+    const int n_items = nt << ch_shift;                            // <= 32: items warp and warp + 16
+    const int it0 = warp, it1 = warp + kWarps;
     float a0[32], a1[32];
-    auto request = [&](int it0, int it1) {
+    {
       const float* P0 = proj + (int64_t(head0 + t0 + (it0 >> ch_shift)) * p.d + (it0 & (chunks - 1)) * 32) * p.r + lane;
       const float* P1 = proj + (int64_t(head0 + t0 + (it1 >> ch_shift)) * p.d + (it1 & (chunks - 1)) * 32) * p.r + lane;
 #pragma unroll
       for (int cc = 0; cc < 32; ++cc) a0[cc] = (it0 < n_items) ? P0[cc * 32] : 0.f;
 #pragma unroll
       for (int cc = 0; cc < 32; ++cc) a1[cc] = (it1 < n_items) ? P1[cc * 32] : 0.f;
-    };
-    auto multiply = [&](int it, const float (&av)[32]) {
-      if (it >= n_items) return;
-      const float* qs = sm->qsum + (it >> ch_shift) * 128 + (it & (chunks - 1)) * 32;
-      float acc = 0.f;
-#pragma unroll
-      for (int cc = 0; cc < 32; ++cc) acc = fmaf(qs[cc], av[cc], acc);
-      sm->upart[it * 32 + lane] = acc;
-    };
-    request(warp, warp + WARPS);
+    }
     for (int i = tid; i < (nt << d_shift); i += kThreads) {
       const int tt = i >> d_shift, c = i & (p.d - 1);
       const int64_t at = (int64_t(rs.b) * p.Hq + int64_t(head0 + t0 + tt) * p.rho) * p.d + c;
@@ -166,12 +153,19 @@ __device__ void build_queries(const Problem& p, const void* q, const float* __re
       sm->qsum[tt * 128 + c] = s;
     }
     __syncthreads();
-    multiply(warp, a0);
-    multiply(warp + WARPS, a1);
-    for (int base = warp + 2 * WARPS; base < n_items; base += 2 * WARPS) {
-      request(base, base + WARPS);
-      multiply(base, a0);
-      multiply(base + WARPS, a1);
+    if (it0 < n_items) {
+      const float* qs = sm->qsum + (it0 >> ch_shift) * 128 + (it0 & (chunks - 1)) * 32;
+      float acc = 0.f;
+#pragma unroll
+      for (int cc = 0; cc < 32; ++cc) acc = fmaf(qs[cc], a0[cc], acc);
+      sm->upart[it0 * 32 + lane] = acc;
+    }
+    if (it1 < n_items) {
+      const float* qs = sm->qsum + (it1 >> ch_shift) * 128 + (it1 & (chunks - 1)) * 32;
+      float acc = 0.f;
+#pragma unroll
+      for (int cc = 0; cc < 32; ++cc) acc = fmaf(qs[cc], a1[cc], acc);
+      sm->upart[it1 * 32 + lane] = acc;
     }
     __syncthreads();
     if (tid < kCols * 32) {
@@ -191,15 +185,10 @@ __device__ void build_queries(const Problem& p, const void* q, const float* __re
 
 // FP8: the metadata is E4M3 (rows of 32 bytes, 64 per tile); every value converts to fp16 exactly, so
 // the product below is the same with twice the rows per byte.
-// LIGHT: 8 warps and no shared-memory histogram (every score is counted in global memory), so that a CTA
-// takes less than half an SM and the scorer can run beside the attention's gather (kvswap_decode_step).
-template <int GS, bool FUSED, bool FP8, bool LIGHT>  // GS = log2(G), 0..5
-__global__ void __launch_bounds__((LIGHT ? kWarpsLight : kWarpsFull) * 32, LIGHT ? 2 : 1)
+template <int GS, bool FUSED, bool FP8>              // GS = log2(G), 0..5
+__global__ void __launch_bounds__(kThreads, 1)
 score_stream_kernel(Problem p, StreamArgs a) {
   constexpr int g_shift = GS;
-  constexpr int kWarps = LIGHT ? kWarpsLight : kWarpsFull;
-  constexpr int kThreads = kWarps * 32;
-  using Smem = SmemT<kWarps, !LIGHT>;
   constexpr int kTileRows = Tile<FP8>::kRows;
   constexpr int kRowBytes = Tile<FP8>::kRowBytes;
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -211,7 +200,7 @@ score_stream_kernel(Problem p, StreamArgs a) {
     for (int s = 0; s < kDepth; ++s) mbar_init(smem_addr(&sm->full[warp * kDepth + s]), 1);
     mbar_init_fence();
   }
-  if (!LIGHT && a.top_hist != nullptr) {
+  if (a.top_hist != nullptr) {
     uint4* H = reinterpret_cast<uint4*>(sm->hist);
     for (int i = threadIdx.x; i < kHistWords / 4; i += kThreads) H[i] = make_uint4(0u, 0u, 0u, 0u);
   }
@@ -260,7 +249,7 @@ score_stream_kernel(Problem p, StreamArgs a) {
   const bool settled = FUSED && (p.flags & KVSWAP_INPUTS_SETTLED) != 0;
   if (!settled) pdl_wait();
   if constexpr (FUSED) {
-    for (int s = 0; s < n_sets; ++s) build_queries<kWarps>(p, a.q, a.proj, row_set(p, rest0 + s, a.n_sub), sm, sm->urow[s]);
+    for (int s = 0; s < n_sets; ++s) build_queries(p, a.q, a.proj, row_set(p, rest0 + s, a.n_sub), sm, sm->urow[s]);
   }
   if (settled) pdl_wait();
   pdl_trigger();
@@ -344,7 +333,7 @@ score_stream_kernel(Problem p, StreamArgs a) {
       if (a.top_hist != nullptr) {
         my_hist = a.top_hist + prob * (kKeyTopBins / 2);
         const int col = (c_rest - rest0) * ns_cols + rq;
-        my_col = (!LIGHT && scope_ok && col < kCols) ? col : -1;
+        my_col = (scope_ok && col < kCols) ? col : -1;
       }
     }
     if (++c_tile == a.tiles_per_row) { c_tile = 0; ++c_rest; }
@@ -416,7 +405,7 @@ score_stream_kernel(Problem p, StreamArgs a) {
   }
 
   // ---- the CTA's counts join the global histograms --------------------------------------------------------
-  if (!LIGHT && a.top_hist != nullptr) {
+  if (a.top_hist != nullptr) {
     __syncthreads();
     for (int i = threadIdx.x; i < kHistWords / 4; i += kThreads) {
       const uint4 v = reinterpret_cast<const uint4*>(sm->hist)[i];
@@ -444,7 +433,6 @@ struct Plan {
   bool fused;
   bool counts;
   bool fp8;
-  bool light;
 };
 
 // Launch geometry of the streaming scorer for `p`; false when the shape does not take it.
@@ -465,34 +453,27 @@ bool plan(const Problem& p, Plan* pl) {
   pl->fp8 = fp8;
   pl->g_shift = g_shift;
   pl->tiles_per_row = int(tiles_per_row); pl->n_sub = n_sub; pl->n_rests = int(n_rests);
-  // Light mode (p.scorer_ctas > 0): that many CTAs of 8 warps, each less than half an SM, beside the
-  // attention's CTAs.  Else one CTA of 16 warps per SM.
-  pl->light = p.scorer_ctas > 0;
-  const int warps_per_cta = pl->light ? kWarpsLight : kWarpsFull;
-  const int max_ctas = pl->light ? p.scorer_ctas : kNumSMs;
-  // When the row sets divide the CTAs (almost) evenly every row set gets its own CTAs, so that no CTA
-  // works for two of them; otherwise all CTAs share the items as one contiguous range.
-  const int per_set = int(max_ctas / std::max<int64_t>(1, n_rests));
-  if (n_rests <= max_ctas && n_rests * per_set * 20 >= int64_t(max_ctas) * 19 && tiles_per_row >= int64_t(per_set) * warps_per_cta) {
+  // One CTA per SM.  When the row sets divide the SMs (almost) evenly every row set gets its own CTAs,
+  // so that no CTA works for two of them; otherwise all CTAs share the items as one contiguous range.
+  const int per_set = int(kNumSMs / std::max<int64_t>(1, n_rests));
+  if (n_rests <= kNumSMs && n_rests * per_set * 20 >= int64_t(kNumSMs) * 19 && tiles_per_row >= int64_t(per_set) * kWarps) {
     pl->vset_items = int(tiles_per_row);
     pl->ctas_per_vset = per_set;
     pl->ctas = int(n_rests) * per_set;
   } else {
     pl->vset_items = int(items);
-    pl->ctas_per_vset = int(std::max<int64_t>(1, std::min<int64_t>(max_ctas, (items + warps_per_cta - 1) / warps_per_cta)));
+    pl->ctas_per_vset = int(std::max<int64_t>(1, std::min<int64_t>(kNumSMs, (items + kWarps - 1) / kWarps)));
     pl->ctas = pl->ctas_per_vset;
   }
-  const int warps = pl->ctas_per_vset * warps_per_cta;
+  const int warps = pl->ctas_per_vset * kWarps;
   pl->base = pl->vset_items / warps;
   pl->rem = pl->vset_items % warps;
   // The CTA builds the low-rank queries itself when it touches few row sets and the adapter has the
-  // layout build_queries() reads (r = 32 columns, d a power of two from 32 to 128).
-  const int64_t cta_items = int64_t(pl->base + 1) * warps_per_cta;
+  // layout build_queries() reads (r = 32 columns, d a multiple of 32 up to 128).
+  const int64_t cta_items = int64_t(pl->base + 1) * kWarps;
   const int64_t sets_touched = (cta_items + tiles_per_row - 1) / tiles_per_row + 1;
   pl->fused = p.r == 32 && (p.d == 32 || p.d == 64 || p.d == 128) && sets_touched <= kMaxSets;
-  // a CTA's counts stay below 2^16 per shared-memory counter (the light scorer has none)
-  pl->counts = pl->light || (pl->base + 1) * warps_per_cta <= kMaxTilesPerCta;
-  if (pl->light && !pl->fused) return false;
+  pl->counts = (pl->base + 1) * kWarps <= kMaxTilesPerCta;   // a CTA's counts stay below 2^16 per counter
   return true;
 }
 
@@ -515,29 +496,27 @@ cudaError_t launch_score_stream(const Problem& p, const void* q, const float* pr
   a.vset_items = pl.vset_items; a.ctas_per_vset = pl.ctas_per_vset; a.base = pl.base; a.rem = pl.rem;
   a.meta_scale = exp2f(float(p.meta_exp));
   a.err = err;
-  auto go = [&](auto kern, size_t smem, int threads) -> cudaError_t {
+  const size_t smem = sizeof(Smem) + 128;
+  auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
-    return launch_pdl(kern, dim3(pl.ctas), dim3(threads), smem, st, p, a);
+    return launch_pdl(kern, dim3(pl.ctas), dim3(kThreads), smem, st, p, a);
   };
-  auto go_gs = [&](auto fused, auto fp8, auto light) -> cudaError_t {
-    constexpr bool F = decltype(fused)::value, E = decltype(fp8)::value, Lt = decltype(light)::value;
-    constexpr int kW = Lt ? kWarpsLight : kWarpsFull;
-    const size_t smem = sizeof(SmemT<kW, !Lt>) + 128;
+  auto go_gs = [&](auto fused, auto fp8) -> cudaError_t {
+    constexpr bool F = decltype(fused)::value, E = decltype(fp8)::value;
     switch (pl.g_shift) {
-      case 0: return go(score_stream_kernel<0, F, E, Lt>, smem, kW * 32);
-      case 1: return go(score_stream_kernel<1, F, E, Lt>, smem, kW * 32);
-      case 2: return go(score_stream_kernel<2, F, E, Lt>, smem, kW * 32);
-      case 3: return go(score_stream_kernel<3, F, E, Lt>, smem, kW * 32);
-      case 4: return go(score_stream_kernel<4, F, E, Lt>, smem, kW * 32);
-      default: return go(score_stream_kernel<5, F, E, Lt>, smem, kW * 32);
+      case 0: return go(score_stream_kernel<0, F, E>);
+      case 1: return go(score_stream_kernel<1, F, E>);
+      case 2: return go(score_stream_kernel<2, F, E>);
+      case 3: return go(score_stream_kernel<3, F, E>);
+      case 4: return go(score_stream_kernel<4, F, E>);
+      default: return go(score_stream_kernel<5, F, E>);
     }
   };
   using T = std::true_type;
   using N = std::false_type;
-  if (pl.light) return pl.fp8 ? go_gs(T(), T(), T()) : go_gs(T(), N(), T());
-  if (pl.fused) return pl.fp8 ? go_gs(T(), T(), N()) : go_gs(T(), N(), N());
-  return pl.fp8 ? go_gs(N(), T(), N()) : go_gs(N(), N(), N());
+  if (pl.fused) return pl.fp8 ? go_gs(T(), T()) : go_gs(T(), N());
+  return pl.fp8 ? go_gs(N(), T()) : go_gs(N(), N());
 }
 
 }  // namespace kvswap

@@ -652,7 +652,7 @@ void plan_sparse_decode(const Problem& p, Workspace* w) {
   // Cost of a split factor s, in chunk times of the slowest CTA: waves * (chunks per CTA + the
   // fixed part of a CTA -- first index fetch, first rows, merge -- worth about 14 chunks), with
   // 2 CTAs per SM resident; at least two chunks per warp and split.
-  const int64_t slots = p.attn_slots > 0 ? p.attn_slots : int64_t(kNumSMs) * 2;   // fewer when the scorer runs beside it
+  const int64_t slots = int64_t(kNumSMs) * 2;
   const int64_t max_splits = std::min<int64_t>(256, std::max<int64_t>(1, n_chunks / (2 * kWarps)));
   int64_t best = 1, best_cost = INT64_MAX;
   for (int64_t s = 1; s <= max_splits; ++s) {

@@ -280,10 +280,8 @@ cudaError_t launch_topk_select(const Problem& p, const float* scores, int32_t* g
 
 namespace {
 
-// MINB = 2 caps the kernel at 32 registers per thread (a few spills), so that its CTAs fit beside the
-// attention's when the predictor and the attention share the GPU.
-template <int P, int MINB>
-__global__ void __launch_bounds__(kPartThreads, MINB)
+template <int P>
+__global__ void __launch_bounds__(kPartThreads)
 topk_parts_kernel(Problem p, const float* __restrict__ scores, uint32_t* __restrict__ top_hist,
                   int32_t* __restrict__ group_idx, int32_t* __restrict__ n_selected) {
   topk_parts_body<P>(p, scores, top_hist, group_idx, n_selected, blockIdx.x, blockIdx.y, gridDim.y);
@@ -322,9 +320,7 @@ cudaError_t launch_topk_parts(const Problem& p, const float* scores, uint32_t* t
   if (P == 0) return cudaErrorInvalidValue;
   const dim3 grid(P, p.B * p.S), block(kPartThreads);
   auto go = [&](auto kern) { return launch_pdl(kern, grid, block, 0, st, p, scores, top_hist, group_idx, n_selected); };
-  if (p.scorer_ctas > 0)
-    return P == 1 ? go(topk_parts_kernel<1, 2>) : P == 2 ? go(topk_parts_kernel<2, 2>) : go(topk_parts_kernel<4, 2>);
-  return P == 1 ? go(topk_parts_kernel<1, 1>) : P == 2 ? go(topk_parts_kernel<2, 1>) : go(topk_parts_kernel<4, 1>);
+  return P == 1 ? go(topk_parts_kernel<1>) : P == 2 ? go(topk_parts_kernel<2>) : go(topk_parts_kernel<4>);
 }
 
 cudaError_t launch_combine_select(const Problem& p, const float* scores, uint32_t* top_hist, int32_t* group_idx,
