@@ -62,6 +62,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="override L (debugging only; reported)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-secondary", action="store_true", help="skip the config-5-per-head and config-4 legs")
+    ap.add_argument("--min-calls", type=int, default=None,
+                    help="launches per per-call figure (default 2000; fewer only for runs under a profiler)")
     return ap.parse_args()
 
 
@@ -235,13 +237,14 @@ def cpu_baseline(wl, dw, meta_heads, scope_name, rt):
 MIN_CALLS = 2000          # launches of a call timed per figure, whatever --steps says
 
 
-def graph_call_us(torch, fns, min_calls=MIN_CALLS):
+def graph_call_us(torch, fns, min_calls=None):
     """Average duration (us) of the calls `fns` (a list: one per layer, each reading another layer's
     buffers, so nothing is served from L2) issued back to back on one stream.  The calls are
     captured once into a CUDA graph and the graph is replayed, so the host is not in the loop;
     CUDA events bracket the replays.  Returns (us per call, calls timed)."""
+    min_calls = MIN_CALLS if min_calls is None else min(min_calls, MIN_CALLS)
     side = torch.cuda.Stream()
-    reps = max(1, -(-72 // len(fns)))                       # calls per graph: at least 72
+    reps = max(1, -(-min(72, min_calls) // len(fns)))       # calls per graph: at least 72
     with torch.cuda.stream(side):
         for f in fns:
             f()
@@ -264,8 +267,9 @@ def graph_call_us(torch, fns, min_calls=MIN_CALLS):
     return a.elapsed_time(b) * 1e3 / (replays * per_graph), replays * per_graph
 
 
-def host_call_us(torch, fns, min_calls=MIN_CALLS):
+def host_call_us(torch, fns, min_calls=None):
     """The same calls issued from Python call by call (the host in the loop)."""
+    min_calls = MIN_CALLS if min_calls is None else min(min_calls, MIN_CALLS)
     for f in fns:
         f()
     reps = max(1, -(-min_calls // len(fns)))
@@ -782,7 +786,10 @@ def reuse_buffer_leg(torch, kv, rt, wl, dw, shape, scope, idx, nsel, out, ws, de
 
 
 def main():
+    global MIN_CALLS
     args = parse_args()
+    if args.min_calls is not None:
+        MIN_CALLS = max(1, args.min_calls)
     wl = W.CONFIGS[args.config]
     if args.layers is not None:
         wl = wl.reduced(wl.name + f"-L{args.layers}", layers=args.layers)
