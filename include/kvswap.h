@@ -12,8 +12,8 @@
  *
  * and around them
  *
- *   kvswap_decode_step / _host        one decode step over all layers of a model, the predictor on
- *                                     an internal stream ahead of the attention (Sec. 4.3, 4.4)
+ *   kvswap_decode_step / _host        one decode step over all layers of a model, each layer predicted
+ *                                     one layer ahead of its attention (Sec. 4.3, 4.4)
  *   kvswap_append_kv / _append_step   a generated token joins the rolling buffer; a completed
  *                                     group is flushed into the compact cache      (Sec. 4.4.1)
  *   kvswap_reuse_* , kvswap_decode_step_tiered, kvswap_append_step_tiered
@@ -34,8 +34,8 @@
  *
  * General conventions
  *  - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
- *    The library never allocates, frees or keeps device memory (kvswap_decode_step creates one
- *    stream and a set of events per device on its first call), and never synchronises: work is
+ *    The library never allocates, frees or keeps device memory (kvswap_decode_step_tiered creates
+ *    one stream and a set of events per device on its first call), and never synchronises: work is
  *    enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream) and the
  *    returned status covers host-side validation and launch errors only.
  *  - Tensors are row-major with a dense last dimension; K, V and the metadata take explicit
@@ -258,9 +258,10 @@ int kvswap_sparse_decode_static(const kvswap_shape* shape, const void* q, const 
 /*
  * Per-layer tensors of a model with L layers that all share one kvswap_shape.  Each member is a
  * HOST array of L DEVICE pointers: K[l], V[l] are [B, H_kv, N, d]; meta[l] is [B, H_m, N, r];
- * proj[l] is [H_kv, d, r] fp32.  max_lookahead bounds how many layers kvswap_decode_step's
- * predictor may run ahead of its attention: 1 = layer l is predicted while layer l-1 is attended
- * (what a model allows, whose layer-l prediction needs the input of layer l-1); 0 = no limit.
+ * proj[l] is [H_kv, d, r] fp32.  max_lookahead bounds how many layers the predictor stream of
+ * kvswap_decode_step_tiered may run ahead of its attention: 1 = layer l is predicted while layer
+ * l-1 is attended (what a model allows, whose layer-l prediction needs the input of layer l-1);
+ * 0 = no limit.  kvswap_decode_step always predicts exactly one layer ahead and ignores the value.
  * Negative values are KVSWAP_ERR_SHAPE.
  */
 typedef struct {
@@ -349,16 +350,16 @@ int kvswap_append_step(const kvswap_shape* shape, const kvswap_layers* layers, c
  *   group_idx  [L, B, S, M] int32, n_selected [L, B, S] int32: the selections of this step, kept
  *              per layer so that the caller can compare consecutive steps (Sec. 4.4.2).
  * `ws` is shared by all layers (size: kvswap_workspace_bytes).  probe_opt may be NULL.
- * The call overlaps prediction and attention as the paper's runtime does (Sec. 4.3 "Online
- * prediction", Sec. 4.4): the predictor (kvswap_score_select's kernels) runs on an internal
- * stream, at most layers->max_lookahead layers ahead of the attention (kvswap_sparse_decode's
- * kernels) on `cuda_stream`; all L queries being given, no data dependency forbids it.  The
- * internal stream is ordered after the work already in `cuda_stream` and has joined it again
- * when the step's last kernel is in it, so the caller synchronises `cuda_stream` only.  The
- * internal stream and its events are created on a device's first call (later calls allocate
- * nothing) and calls are serialised by a process-wide lock.  Results are identical to calling
- * kvswap_score_select and kvswap_sparse_decode layer by layer.  A probe's ev_begin and ev_mid
- * are recorded on the internal stream, ev_end on `cuda_stream`.
+ * The call orders prediction and attention as the paper's runtime does (Sec. 4.3 "Online
+ * prediction", Sec. 4.4): layer l + 1 is scored before layer l is attended and its TopK follows
+ * that attention, i.e. the predictor is exactly one layer ahead -- what a model allows whose
+ * layer-(l+1) prediction is formed from the input of layer l.  Everything is enqueued on
+ * `cuda_stream` as programmatic dependent launches (a kernel's set-up and first fetches overlap
+ * the tail of the kernel before it); the call keeps no state, creates nothing and takes no lock.
+ * Results are identical to calling kvswap_score_select and kvswap_sparse_decode layer by layer.
+ * A probe's events are recorded on `cuda_stream`: ev_begin before the layer's scorer, ev_mid
+ * after its TopK, ev_end after its attention (the attention of the layer before lies between
+ * ev_begin and ev_mid).
  */
 int kvswap_decode_step(const kvswap_shape* shape, const kvswap_layers* layers, const void* q,
                        float* out, float* lse_opt, int32_t* group_idx, int32_t* n_selected,

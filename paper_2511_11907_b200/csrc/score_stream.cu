@@ -1,9 +1,11 @@
 // K2, streaming tensor-core scorer: low-rank query (Eq. 1), token scoring, head aggregation and
-// group ReduceMax (Sec. 4.3) for fp16 metadata rows of 64 bytes (r = 32) that are dense in memory,
-// G a power of two <= 32 and one metadata term per score.
+// group ReduceMax (Sec. 4.3) for metadata rows of rank 32 that are dense in memory -- fp16 rows of
+// 64 bytes, or 8-bit E4M3 rows of 32 bytes whose values convert to fp16 exactly and whose common
+// power-of-two scale is applied to the finished score -- G a power of two <= 32 and one metadata
+// term per score.
 //
 // One persistent CTA per SM, 16 warps.  Work item = (sequence b, metadata head hm, block of 8
-// scopes, tile of 32 rows); items are numbered with the tile fastest, a "row set" is the items of
+// scopes, 2 KB tile of 32 fp16 or 64 E4M3 rows); items are numbered with the tile fastest, a "row set" is the items of
 // one (b, hm, scope block).  Every warp takes an equal contiguous share of tiles and pulls them
 // into its own ring of shared-memory stages with bulk asynchronous copies (cp.async.bulk +
 // mbarrier, bounded waits), kDepth tiles in flight per warp; the first tiles are requested before

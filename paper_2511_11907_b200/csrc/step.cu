@@ -1,7 +1,8 @@
-// C-ABI entry points that serve all layers of a model in one call: the decode step with the
-// predictor on a stream of its own (over HBM-resident stores or over reuse buffers in front of a
-// slow tier) and the append steps.  kvswap_decode_step keeps one internal stream and a set of
-// events per device; nothing else here keeps state.
+// C-ABI entry points that serve all layers of a model in one call: the decode step over
+// HBM-resident stores (one stream, each layer predicted one layer ahead of its attention), the
+// decode step over reuse buffers in front of a slow tier (the predictor on a stream of its own)
+// and the append steps.  The tiered step keeps one internal stream and a set of events per device;
+// nothing else here keeps state.
 #include <algorithm>
 #include <mutex>
 #include <vector>
