@@ -90,12 +90,18 @@ static bool counts_top_digit(const Problem& p) {
   return !(p.flags & KVSWAP_SCORE_SOFTMAX) && hist_capable(p) && score_stream_counts_top_digit(p) && topk_parts_supported(p);
 }
 
+bool query_ahead_supported(const Problem& p) {
+  return p.NG > 0 && !(p.flags & KVSWAP_SCORE_SOFTMAX) && score_stream_supported(p) && score_stream_fuses_query(p) &&
+         counts_top_digit(p);
+}
+
 void plan_workspace(const Problem& p, Workspace* w) {
   plan_sparse_decode(p, w);
 
   size_t off = 256;  // first 256 bytes reserved
   w->off_hist = off;     off += hist_capable(p) ? align256(size_t(p.B) * p.S * (sizeof(uint16_t) * kKeyTopBins + sizeof(uint32_t))) : 0;
-  w->off_uq = off;       off += align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
+  w->uq_bytes = align256(sizeof(float) * size_t(p.B) * p.Su * p.r);
+  w->off_uq = off;       off += 2 * w->uq_bytes;
   w->off_scores = off;   off += align256(sizeof(float) * size_t(p.B) * p.S * workspace_score_pitch(p));
   w->off_partial = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * w->splits * (p.d + 2));
   w->off_softmax = off;  off += align256(sizeof(float) * size_t(p.B) * p.Hq * (size_t(p.r) + 2 * size_t(score_softmax_chunks(p))));
@@ -126,9 +132,9 @@ int check_score_select(const kvswap_shape* shape, const void* q, const float* pr
 // group scores (and, where that path exists, the leading-digit histograms) in the workspace or the
 // caller's buffer, and the TopK over them.  A step may put other work between the two.
 cudaError_t score_launch(const Problem& p_in, const Workspace& w, const void* q, const float* proj, const void* meta,
-                         float* group_scores_opt, void* ws, cudaStream_t stream) {
+                         float* group_scores_opt, void* ws, cudaStream_t stream, int uq_ahead) {
   char* base = static_cast<char*>(ws);
-  float* uq = reinterpret_cast<float*>(base + w.off_uq);
+  float* uq = reinterpret_cast<float*>(base + w.off_uq + (uq_ahead > 0 ? w.uq_bytes : 0));
   float* scores = group_scores_opt ? group_scores_opt : reinterpret_cast<float*>(base + w.off_scores);
   Problem p = p_in;
   p.score_pitch = group_scores_opt ? p.NG : workspace_score_pitch(p);     // a caller's buffer is dense [B, S, NG]
@@ -142,6 +148,10 @@ cudaError_t score_launch(const Problem& p_in, const Workspace& w, const void* q,
     // where it can and counts the leading digits of its scores for the TopK that follows
     uint32_t* top_hist = counts_top_digit(p) ? reinterpret_cast<uint32_t*>(base + w.off_hist) : nullptr;
     const bool fused = score_stream_fuses_query(p);
+    if (uq_ahead >= 0) {                                                  // the queries are in the workspace already
+      if (!fused) return cudaErrorInvalidValue;
+      return launch_score_stream(p, nullptr, proj, uq, meta, scores, top_hist, static_cast<uint32_t*>(ws), stream);
+    }
     cudaError_t e = fused ? cudaSuccess : launch_lowrank_query(p, q, proj, uq, stream);
     if (e != cudaSuccess) return e;
     return launch_score_stream(p, fused ? q : nullptr, proj, uq, meta, scores, top_hist, static_cast<uint32_t*>(ws),
@@ -168,14 +178,17 @@ cudaError_t select_launch(const Problem& p_in, const Workspace& w, int32_t* grou
 // when the select of this shape has no such kernel (the caller then launches the two separately).
 bool select_with_combine_launch(const Problem& p_in, const Workspace& w, int32_t* group_idx, int32_t* n_selected,
                                 void* ws, const float* partial, float* out, float* lse, int splits, int n_rows, int d,
-                                cudaStream_t stream, cudaError_t* result) {
+                                cudaStream_t stream, cudaError_t* result, const void* q_ahead,
+                                const float* proj_ahead, int uq_ahead) {
   Problem p = p_in;
   p.score_pitch = workspace_score_pitch(p);
   if (!(p.NG > 0 && score_stream_supported(p) && counts_top_digit(p))) return false;
   char* base = static_cast<char*>(ws);
+  float* uq = reinterpret_cast<float*>(base + w.off_uq + (uq_ahead > 0 ? w.uq_bytes : 0));
+  const bool ahead = q_ahead != nullptr && uq_ahead >= 0 && score_stream_fuses_query(p);
   *result = launch_combine_select(p, reinterpret_cast<float*>(base + w.off_scores),
                                   reinterpret_cast<uint32_t*>(base + w.off_hist), group_idx, n_selected, partial, out, lse,
-                                  splits, n_rows, d, stream);
+                                  splits, n_rows, d, ahead ? q_ahead : nullptr, proj_ahead, uq, stream);
   return true;
 }
 

@@ -32,7 +32,8 @@ struct Problem {
 
 // Partition of the caller's workspace (byte offsets, each 256-byte aligned).
 struct Workspace {
-  size_t off_uq;       // float [B, Su, r]       summed low-rank queries
+  size_t off_uq;       // float [2][B, Su, r]    summed low-rank queries; two buffers of uq_bytes (a decode step alternates)
+  size_t uq_bytes;
   size_t off_scores;   // float [B, S, NG]       group scores R (when the caller passes no buffer)
   size_t off_hist;     // uint16 [B, S, 4096] + uint32 [B, S]  leading-digit histograms of the group scores' keys and tickets, zero between calls
   size_t off_partial;  // float [B, Hq, splits, d + 2]  split-K partials (m, l, acc[d])
@@ -82,8 +83,8 @@ cudaError_t launch_lowrank_query(const Problem& p, const void* q, const float* p
 cudaError_t launch_score_pool(const Problem& p, const float* uq, const void* meta, float* scores,
                               uint32_t* err, cudaStream_t st);
 // The streaming tensor-core scorer (score_stream.cu) for fp16 metadata rows of 64 bytes.  Where it
-// builds the low-rank queries itself it takes q and proj (uq unused), else uq from
-// launch_lowrank_query.  `top_hist` (may be NULL): per (sequence, scope) a histogram of the leading
+// builds the low-rank queries itself it takes q and proj (uq unused), else -- or when q is NULL --
+// uq [B, Su, r] from launch_lowrank_query or from the kernel of launch_combine_select.  `top_hist` (may be NULL): per (sequence, scope) a histogram of the leading
 // 12 bits of the group scores' keys (4096 16-bit counters, two per word) followed, after all
 // histograms, by one ticket word per (sequence, scope).  Everything is zero on entry; the scorer
 // counts, and launch_topk_parts, which starts from the counts, leaves everything zero again.
@@ -106,10 +107,17 @@ cudaError_t launch_sparse_decode(const Problem& p, const Workspace& w, const voi
 cudaError_t launch_combine_only(const Problem& p, const Workspace& w, const float* partial, float* out, float* lse,
                                 cudaStream_t st);
 // launch_topk_parts for problem `p` and, in the same launch, the merge of `n_rows` rows of split-K
-// partials [n_rows, splits, d + 2] (of whatever attention produced them) into out / lse.
+// partials [n_rows, splits, d + 2] (of whatever attention produced them) into out / lse.  With
+// q_ahead != NULL the launch also builds the summed low-rank queries of another layer of the same shape
+// (its q and proj) into uq_ahead [B, Su, r], for a streaming scorer that is enqueued next: the bits are
+// those the scorer would build itself.  Only where score_stream_fuses_query(p).
 cudaError_t launch_combine_select(const Problem& p, const float* scores, uint32_t* top_hist, int32_t* group_idx,
                                   int32_t* n_selected, const float* partial, float* out, float* lse, int splits,
-                                  int n_rows, int d, cudaStream_t st);
+                                  int n_rows, int d, const void* q_ahead, const float* proj_ahead, float* uq_ahead,
+                                  cudaStream_t st);
+// Row sets of the streaming scorer for `p` (0 when it does not take the shape) and scope blocks per
+// (sequence, metadata head): the arguments of row_set() in lowrank_query.cuh.
+void score_stream_row_sets(const Problem& p, int* n_rests, int* n_sub);
 
 // Launch with programmatic stream serialisation: the kernel may begin (up to its
 // griddepcontrol.wait) while the previous kernel in the stream is still draining.

@@ -43,6 +43,7 @@
 
 #include "async_copy.cuh"
 #include "common.cuh"
+#include "lowrank_query.cuh"
 #include "topk_keys.cuh"
 
 namespace kvswap {
@@ -54,10 +55,10 @@ template <bool FP8> struct Tile {
   static constexpr int kRowBytes = FP8 ? 32 : 64;
   static constexpr int kRows = kTileBytes / kRowBytes;
 };
-constexpr int kWarps = 16;
+constexpr int kWarps = kQueryWarps;                       // 16
 constexpr int kThreads = kWarps * 32;
 constexpr int kDepth = 4;
-constexpr int kCols = 8;                                  // scores per metadata row and instruction
+constexpr int kCols = kQueryCols;                         // scores per metadata row and instruction
 constexpr int kHistWords = kCols * kKeyTopBins / 2;       // two 16-bit counters per word
 constexpr int kMaxSets = 4;                               // row sets one CTA may touch when it builds the queries itself
 constexpr int kMaxTilesPerCta = 65535 / 64;                // bound that keeps a 16-bit counter from overflowing (64 rows, G = 1)
@@ -66,8 +67,8 @@ struct Smem {
   unsigned char tiles[kWarps * kDepth * kTileBytes];      // 128 KB of stages
   uint32_t hist[kHistWords];                              // 64 KB
   unsigned long long full[kWarps * kDepth];
-  float qsum[8 * 128];                                    // summed queries of up to 8 KV heads
-  float upart[32 * 32];                                   // partial products, [item][column]
+  float qsum[kQuerySumFloats];                            // scratch of build_queries
+  float upart[kQueryPartFloats];
   float urow[kMaxSets][kCols * 32];                       // summed low-rank queries per row set of the CTA
 };
 
@@ -95,94 +96,6 @@ __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1
 
 __device__ __forceinline__ uint32_t pack_half2(__half lo, __half hi) {
   return uint32_t(__half_as_ushort(lo)) | (uint32_t(__half_as_ushort(hi)) << 16);
-}
-
-__device__ __forceinline__ float load_q(const void* q, int dtype, int64_t i) {
-  if (dtype == KVSWAP_F32) return static_cast<const float*>(q)[i];
-  if (dtype == KVSWAP_BF16) return __bfloat162float(static_cast<const __nv_bfloat16*>(q)[i]);
-  return __half2float(static_cast<const __half*>(q)[i]);
-}
-
-// (sequence, metadata head, scope block) of a row set.
-struct RowSet { int b, hm, sub; };
-__device__ __forceinline__ RowSet row_set(const Problem& p, int rest, int n_sub) {
-  const int hm_count = (p.Hm == 1) ? 1 : p.Hkv;
-  const int bh = rest / n_sub;
-  return RowSet{bh / hm_count, bh % hm_count, rest % n_sub};
-}
-
-// Summed low-rank queries of one row set into urow[8][32] (rows beyond the set's scopes are zero).
-// The KV heads that feed the rows are taken eight at a time.  An item is 32 channels of one head:
-// a warp multiplies the head's summed query by the adapter rows (coalesced 128-byte reads of A_g);
-// it requests the adapter rows of its (at most two) items first, then the CTA sums the query
-// heads into shared memory, so that both loads share one round trip.  The partial products are
-// added in a fixed order.  All threads call.
-__device__ void build_queries(const Problem& p, const void* q, const float* __restrict__ proj, RowSet rs,
-                              Smem* sm, float* urow) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool joint = p.Hm == 1;
-  const bool all_heads = joint && p.scope == KVSWAP_SCOPE_ALL_HEADS;
-  // term t of the row set: (row it adds to, KV head it reads)
-  const int n_terms = all_heads ? p.Hkv : joint ? min(kCols, p.S - rs.sub * kCols) : 1;
-  const int head0 = all_heads ? 0 : joint ? rs.sub * kCols : rs.hm;      // head of term t: head0 + t
-  const bool row_per_term = joint && !all_heads;                          // row of term t: t, else 0
-  const int ch_shift = (p.d == 128) ? 2 : (p.d == 64) ? 1 : 0;            // 32-channel pieces of a head: 4, 2 or 1
-  const int chunks = 1 << ch_shift;
-  const int d_shift = ch_shift + 5;
-  for (int t0 = 0; t0 < n_terms; t0 += 8) {
-    const int nt = min(8, n_terms - t0);
-    const int n_items = nt << ch_shift;                            // <= 32: items warp and warp + 16
-    const int it0 = warp, it1 = warp + kWarps;
-    float a0[32], a1[32];
-    {
-      const float* P0 = proj + (int64_t(head0 + t0 + (it0 >> ch_shift)) * p.d + (it0 & (chunks - 1)) * 32) * p.r + lane;
-      const float* P1 = proj + (int64_t(head0 + t0 + (it1 >> ch_shift)) * p.d + (it1 & (chunks - 1)) * 32) * p.r + lane;
-#pragma unroll
-      for (int cc = 0; cc < 32; ++cc) a0[cc] = (it0 < n_items) ? P0[cc * 32] : 0.f;
-#pragma unroll
-      for (int cc = 0; cc < 32; ++cc) a1[cc] = (it1 < n_items) ? P1[cc * 32] : 0.f;
-    }
-    for (int i = tid; i < (nt << d_shift); i += kThreads) {
-      const int tt = i >> d_shift, c = i & (p.d - 1);
-      const int64_t at = (int64_t(rs.b) * p.Hq + int64_t(head0 + t0 + tt) * p.rho) * p.d + c;
-      float s = 0.f;
-      for (int h0 = 0; h0 < p.rho; h0 += 4) {                      // the loads of four heads go out together
-        float v[4];
-#pragma unroll
-        for (int hh = 0; hh < 4; ++hh) v[hh] = (h0 + hh < p.rho) ? load_q(q, p.q_dtype, at + int64_t(h0 + hh) * p.d) : 0.f;
-        s += (v[0] + v[1]) + (v[2] + v[3]);
-      }
-      sm->qsum[tt * 128 + c] = s;
-    }
-    __syncthreads();
-    if (it0 < n_items) {
-      const float* qs = sm->qsum + (it0 >> ch_shift) * 128 + (it0 & (chunks - 1)) * 32;
-      float acc = 0.f;
-#pragma unroll
-      for (int cc = 0; cc < 32; ++cc) acc = fmaf(qs[cc], a0[cc], acc);
-      sm->upart[it0 * 32 + lane] = acc;
-    }
-    if (it1 < n_items) {
-      const float* qs = sm->qsum + (it1 >> ch_shift) * 128 + (it1 & (chunks - 1)) * 32;
-      float acc = 0.f;
-#pragma unroll
-      for (int cc = 0; cc < 32; ++cc) acc = fmaf(qs[cc], a1[cc], acc);
-      sm->upart[it1 * 32 + lane] = acc;
-    }
-    __syncthreads();
-    if (tid < kCols * 32) {
-      const int row = tid >> 5, j = tid & 31;
-      float s = (t0 == 0) ? 0.f : urow[tid];
-      if (row_per_term) {                                          // the items of term `row`
-        if (row < nt)
-          for (int ch = 0; ch < chunks; ++ch) s += sm->upart[((row << ch_shift) + ch) * 32 + j];
-      } else if (row == 0) {
-        for (int it = 0; it < n_items; ++it) s += sm->upart[it * 32 + j];
-      }
-      urow[tid] = s;
-    }
-    __syncthreads();
-  }
 }
 
 // FP8: the metadata is E4M3 (rows of 32 bytes, 64 per tile); every value converts to fp16 exactly, so
@@ -251,7 +164,7 @@ score_stream_kernel(Problem p, StreamArgs a) {
   const bool settled = FUSED && (p.flags & KVSWAP_INPUTS_SETTLED) != 0;
   if (!settled) pdl_wait();
   if constexpr (FUSED) {
-    for (int s = 0; s < n_sets; ++s) build_queries(p, a.q, a.proj, row_set(p, rest0 + s, a.n_sub), sm, sm->urow[s]);
+    for (int s = 0; s < n_sets; ++s) build_queries<0>(p, a.q, a.proj, row_set(p, rest0 + s, a.n_sub), sm->qsum, sm->upart, sm->urow[s]);
   }
   if (settled) pdl_wait();
   pdl_trigger();
@@ -484,13 +397,21 @@ bool plan(const Problem& p, Plan* pl) {
 bool score_stream_supported(const Problem& p) { Plan pl; return plan(p, &pl); }
 bool score_stream_fuses_query(const Problem& p) { Plan pl; return plan(p, &pl) && pl.fused; }
 bool score_stream_counts_top_digit(const Problem& p) { Plan pl; return plan(p, &pl) && pl.counts; }
+void score_stream_row_sets(const Problem& p, int* n_rests, int* n_sub) {
+  Plan pl;
+  const bool ok = plan(p, &pl);
+  *n_rests = ok ? pl.n_rests : 0;
+  *n_sub = ok ? pl.n_sub : 1;
+}
 
 cudaError_t launch_score_stream(const Problem& p, const void* q, const float* proj, const float* uq, const void* meta,
                                 float* scores, uint32_t* top_hist, uint32_t* err, cudaStream_t st) {
   Plan pl;
   if (!plan(p, &pl)) return cudaErrorInvalidValue;
   if (top_hist != nullptr && !pl.counts) return cudaErrorInvalidValue;
-  if (pl.fused ? (q == nullptr || proj == nullptr) : (uq == nullptr)) return cudaErrorInvalidValue;
+  // With q == NULL the queries come from `uq` even where the kernel could build them.
+  if (q == nullptr) pl.fused = false;
+  if (pl.fused ? (proj == nullptr) : (uq == nullptr)) return cudaErrorInvalidValue;
   StreamArgs a;
   a.q = q; a.proj = proj; a.uq = uq; a.meta = static_cast<const unsigned char*>(meta); a.scores = scores;
   a.top_hist = top_hist;

@@ -190,10 +190,17 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
     shape_settled.flags |= KVSWAP_INPUTS_SETTLED;
     auto ev = [&](void* e) { if (e != nullptr) cudaEventRecord(static_cast<cudaEvent_t>(e), stream); };
     auto probed = [&](int l) { return probe_opt != nullptr && probe_opt->layer == l; };
+    // Where the kernel that merges layer l's partials and selects for layer l + 1 can also form the
+    // summed low-rank queries of layer l + 2 (its combine CTAs idle until the gather has finished),
+    // that layer's scorer finds them in the workspace and goes straight to its tiles.  The workspace
+    // has two query buffers: the scorer of layer l + 1 may still be reading its own.
+    const bool ahead = query_ahead_supported(p);
+    int formed_for = -1;                            // the layer whose queries the last merged launch formed
     auto score = [&](int l) -> int {
       if (probed(l)) ev(probe_opt->ev_begin);
       const void* ql = static_cast<const char*>(q) + size_t(l) * q_bytes;
-      return score_launch(p_settled, w, ql, layers->proj[l], layers->meta[l], nullptr, ws, stream) == cudaSuccess
+      return score_launch(p_settled, w, ql, layers->proj[l], layers->meta[l], nullptr, ws, stream,
+                          formed_for == l ? (l & 1) : -1) == cudaSuccess
                  ? KVSWAP_OK : KVSWAP_ERR_CUDA;
     };
     auto select = [&](int l) -> int {
@@ -218,9 +225,13 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
                                static_cast<uint32_t*>(ws), stream, /*combine=*/false) != cudaSuccess)
         return KVSWAP_ERR_CUDA;
       cudaError_t e = cudaSuccess;
+      const bool form = ahead && l + 2 < L;
+      const void* q_ahead = form ? static_cast<const char*>(q) + size_t(l + 2) * q_bytes : nullptr;
       const bool merged = next && select_with_combine_launch(p_settled, w, group_idx + size_t(l + 1) * idx_elems,
                                                              n_selected + size_t(l + 1) * nsel_elems, ws, partial, out_l,
-                                                             lse_l, w.splits, p.B * p.Hq, p.d, stream, &e);
+                                                             lse_l, w.splits, p.B * p.Hq, p.d, stream, &e, q_ahead,
+                                                             form ? layers->proj[l + 2] : nullptr, (l + 2) & 1);
+      if (merged && form && e == cudaSuccess) formed_for = l + 2;
       if (!merged) {
         e = launch_combine_only(p, w, partial, out_l, lse_l, stream);
       }

@@ -11,6 +11,7 @@
 //   topk_select_kernel        longer rows: keys in shared memory (or re-read), 8-bit digits.
 #include "async_copy.cuh"
 #include "combine.cuh"
+#include "lowrank_query.cuh"
 #include "common.cuh"
 #include "topk_keys.cuh"
 #include "topk_parts.cuh"
@@ -287,26 +288,47 @@ topk_parts_kernel(Problem p, const float* __restrict__ scores, uint32_t* __restr
   topk_parts_body<P>(p, scores, top_hist, group_idx, n_selected, blockIdx.x, blockIdx.y, gridDim.y);
 }
 
-// The select of one layer beside the split-K combine of another in one launch: the first
-// P * problems CTAs select, the rest merge 1024 / D (sequence, head) rows of partials each.  Both are
-// short, latency-bound kernels; side by side they cost the longer of the two, and one launch gap.
+// Rows of partials one CTA merges, D threads and one named barrier (1 .. 14) each; barrier 15 is the
+// query build's.
+template <int D> constexpr int kCombineRows = (kPartThreads / D < 14) ? kPartThreads / D : 14;
+
+// The select of one layer beside the split-K combine of another in one launch: the first CTAs merge
+// kCombineRows (sequence, head) rows of partials each, the other P * problems CTAs select.  Both are short,
+// latency-bound kernels; side by side they cost the longer of the two, and one launch gap.
+//
+// The combine CTAs have nothing to do until the gather before them has finished.  With q_ahead they
+// use that time for the summed low-rank queries of the layer whose scorer is enqueued next (row sets
+// cta, cta + n_comb, ..): half of the CTA's threads run the scorer's own build_queries() and store the
+// rows where that scorer looks for them, so that it starts on its tiles as soon as this kernel ends.
 template <int P, int D>
 __global__ void __launch_bounds__(kPartThreads)
 combine_select_kernel(Problem p, const float* __restrict__ scores, uint32_t* __restrict__ top_hist,
                       int32_t* __restrict__ group_idx, int32_t* __restrict__ n_selected, int n_probs,
                       const float* __restrict__ partial, float* __restrict__ out, float* __restrict__ lse, int splits,
-                      int n_rows) {
-  constexpr int kRows = kPartThreads / D;            // rows of partials merged per CTA
-  __shared__ float w_s[kRows][kMaxSplits];
-  __shared__ float norm_s[kRows][2];
-  if (int(blockIdx.x) < P * n_probs) {
-    topk_parts_body<P>(p, scores, top_hist, group_idx, n_selected, int(blockIdx.x) % P, int(blockIdx.x) / P, n_probs);
+                      int n_rows, int n_comb, const void* __restrict__ q_ahead, const float* __restrict__ proj_ahead,
+                      float* __restrict__ uq_ahead, int n_rests, int n_sub) {
+  constexpr int kRows = kCombineRows<D>;             // rows of partials merged per CTA
+  if (int(blockIdx.x) >= n_comb) {
+    const int t = int(blockIdx.x) - n_comb;
+    topk_parts_body<P>(p, scores, top_hist, group_idx, n_selected, t % P, t / P, n_probs);
     return;
   }
+  __shared__ float w_s[kRows][kMaxSplits];
+  __shared__ float norm_s[kRows][2];
+  __shared__ float qsum[kQuerySumFloats], upart[kQueryPartFloats], urow[kQueryCols * 32];
   pdl_trigger();
+  if (q_ahead != nullptr && threadIdx.x < kQueryThreads) {
+    for (int rest = blockIdx.x; rest < n_rests; rest += n_comb) {
+      const RowSet rs = row_set(p, rest, n_sub);
+      build_queries<15>(p, q_ahead, proj_ahead, rs, qsum, upart, urow);
+      store_queries(p, rs, urow, uq_ahead);
+      asm volatile("bar.sync 15, %0;" ::"n"(kQueryThreads) : "memory");       // urow is free for the next row set
+    }
+  }
   pdl_wait();
   const int slot = int(threadIdx.x) / D;
-  const int64_t row = int64_t(int(blockIdx.x) - P * n_probs) * kRows + slot;
+  if (slot >= kRows) return;
+  const int64_t row = int64_t(blockIdx.x) * kRows + slot;
   combine_row<D>(partial, out, lse, splits, row, row < n_rows, int(threadIdx.x) % D, w_s[slot], norm_s[slot], 1 + slot);
 }
 
@@ -325,15 +347,22 @@ cudaError_t launch_topk_parts(const Problem& p, const float* scores, uint32_t* t
 
 cudaError_t launch_combine_select(const Problem& p, const float* scores, uint32_t* top_hist, int32_t* group_idx,
                                   int32_t* n_selected, const float* partial, float* out, float* lse, int splits,
-                                  int n_rows, int d, cudaStream_t st) {
+                                  int n_rows, int d, const void* q_ahead, const float* proj_ahead, float* uq_ahead,
+                                  cudaStream_t st) {
   const int P = plan_topk_parts(p);
   if (P == 0 || (d != 64 && d != 128) || splits > kMaxSplits) return cudaErrorInvalidValue;
+  int n_rests = 0, n_sub = 1;
+  if (q_ahead != nullptr) {
+    if (!score_stream_fuses_query(p) || proj_ahead == nullptr || uq_ahead == nullptr) return cudaErrorInvalidValue;
+    score_stream_row_sets(p, &n_rests, &n_sub);
+  }
   const int n_probs = p.B * p.S;
-  const int rows_per_cta = kPartThreads / d;
-  const dim3 grid(P * n_probs + (n_rows + rows_per_cta - 1) / rows_per_cta), block(kPartThreads);
+  const int rows_per_cta = (d == 128) ? kCombineRows<128> : kCombineRows<64>;
+  const int n_comb = (n_rows + rows_per_cta - 1) / rows_per_cta;
+  const dim3 grid(n_comb + P * n_probs), block(kPartThreads);
   auto go = [&](auto kern) {
     return launch_pdl(kern, grid, block, 0, st, p, scores, top_hist, group_idx, n_selected, n_probs, partial, out, lse,
-                      splits, n_rows);
+                      splits, n_rows, n_comb, q_ahead, proj_ahead, uq_ahead, n_rests, n_sub);
   };
   if (d == 128) return P == 1 ? go(combine_select_kernel<1, 128>) : P == 2 ? go(combine_select_kernel<2, 128>) : go(combine_select_kernel<4, 128>);
   return P == 1 ? go(combine_select_kernel<1, 64>) : P == 2 ? go(combine_select_kernel<2, 64>) : go(combine_select_kernel<4, 64>);

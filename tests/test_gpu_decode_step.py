@@ -1,6 +1,7 @@
-"""kvswap_decode_step (all layers of one decode step in one call, each layer's predictor on an
-internal stream overlapping the previous layer's attention) gives exactly what the per-layer
-calls give.  The per-layer calls themselves are checked against the oracle in test_gpu_parity.py."""
+"""kvswap_decode_step (all layers of one decode step in one call: each layer scored one layer ahead
+of its attention, its TopK merged with the previous layer's split-K combine, the low-rank queries
+of the layer after it formed in the same launch) gives exactly what the per-layer calls give.  The
+per-layer calls themselves are checked against the oracle in test_gpu_parity.py."""
 import pytest
 import torch
 
@@ -61,7 +62,7 @@ def _run_case(wl, meta_heads, scope, lookahead=0):
     assert torch.equal(idx_a, idx_c)
     assert torch.equal(out_a.cpu(), out_host)
 
-    # repeated steps reuse the internal stream and events
+    # repeated steps
     for _ in range(3):
         kv.kvswap_decode_step(dw.shape, dw.layer_tables(lookahead), q, out_b, lse_b, idx_b, nsel_b, ws)
     torch.cuda.synchronize()
@@ -94,6 +95,14 @@ def test_decode_step_over_many_layers(lookahead):
     wl = W.CONFIGS[3].reduced("cfg3-deep", layers=70, batch=1, n_ctx=1024 + 3, top_k=16, calib_rows=1024,
                               n_q_heads=8, n_kv_heads=2)
     _run_case(wl, "joint", W.SCOPE_KV_HEAD, lookahead)
+
+
+@pytest.mark.parametrize("meta_heads", ["joint", "per_head"])
+def test_decode_step_head_dim_64(meta_heads):
+    """d = 64: the merged combine + TopK launch merges 14 rows of partials per CTA, and the low-rank
+    queries formed a layer ahead take two 32-channel pieces per head."""
+    wl = W.CONFIGS[4].reduced("cfg4-d64", layers=4, batch=3, n_ctx=4096 + 19, top_k=40, calib_rows=1024, head_dim=64)
+    _run_case(wl, meta_heads, W.SCOPE_KV_HEAD)
 
 
 def test_decode_step_fp32_wide_rank_per_head():
