@@ -90,6 +90,10 @@ static bool counts_top_digit(const Problem& p) {
   return !(p.flags & KVSWAP_SCORE_SOFTMAX) && hist_capable(p) && score_stream_counts_top_digit(p) && topk_parts_supported(p);
 }
 
+bool select_merges_with_combine(const Problem& p) {
+  return p.NG > 0 && score_stream_supported(p) && counts_top_digit(p);
+}
+
 bool query_ahead_supported(const Problem& p) {
   return p.NG > 0 && !(p.flags & KVSWAP_SCORE_SOFTMAX) && score_stream_supported(p) && score_stream_fuses_query(p) &&
          counts_top_digit(p);
@@ -182,7 +186,7 @@ bool select_with_combine_launch(const Problem& p_in, const Workspace& w, int32_t
                                 const float* proj_ahead, int uq_ahead) {
   Problem p = p_in;
   p.score_pitch = workspace_score_pitch(p);
-  if (!(p.NG > 0 && score_stream_supported(p) && counts_top_digit(p))) return false;
+  if (!select_merges_with_combine(p)) return false;
   char* base = static_cast<char*>(ws);
   float* uq = reinterpret_cast<float*>(base + w.off_uq + (uq_ahead > 0 ? w.uq_bytes : 0));
   const bool ahead = q_ahead != nullptr && uq_ahead >= 0 && score_stream_fuses_query(p);

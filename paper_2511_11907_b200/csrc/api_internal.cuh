@@ -31,6 +31,8 @@ bool select_with_combine_launch(const Problem& p_in, const Workspace& w, int32_t
                                 cudaStream_t stream, cudaError_t* result, const void* q_ahead = nullptr,
                                 const float* proj_ahead = nullptr, int uq_ahead = -1);
 bool query_ahead_supported(const Problem& p);
+// True when select_with_combine_launch has a kernel for this shape's select.
+bool select_merges_with_combine(const Problem& p);
 // Both halves back to back.
 cudaError_t score_select_launch(const Problem& p_in, const Workspace& w, const void* q,
                                 const float* proj, const void* meta, int32_t* group_idx, int32_t* n_selected,

@@ -18,7 +18,7 @@ constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs; grids are sized in multi
 struct Problem {
   int B, N, Hq, Hkv, d, r, Hm, G, M;
   int kv_dtype, meta_dtype, q_dtype, scope;
-  int flags;   // KVSWAP_INPUTS_SETTLED, KVSWAP_SCORE_SOFTMAX
+  int flags;   // KVSWAP_INPUTS_SETTLED, KVSWAP_SCORE_SOFTMAX, kFlag*
   int meta_exp;   // 8-bit metadata stores K_lr * 2^-meta_exp (0 for the other types)
   int64_t kv_sb, kv_sh, kv_sn;
   int64_t meta_sb, meta_sh, meta_sn;
@@ -29,6 +29,15 @@ struct Problem {
   int Su;    // rows of the low-rank query buffer per sequence (see score_pool.cu)
   int score_pitch;   // floats between rows of the group-score buffer: NG in a caller's buffer, padded in the workspace
 };
+
+// Internal flags (never taken from a caller's shape; a decode step sets them).
+// kFlagWaitEarly, on the split-K gather with KVSWAP_INPUTS_SETTLED: the dependency wait comes right after
+// the first fills are requested, and only then may the kernel enqueued behind this one start.
+// kFlagInputsTwoBack, on the TopK enqueued behind such a gather: its scores and counts were complete
+// before the gather's wait returned, i.e. before any of its own CTAs started, and nothing it writes is
+// touched by the gather: it does not wait at all.
+constexpr int kFlagWaitEarly = 1 << 16;
+constexpr int kFlagInputsTwoBack = 1 << 17;
 
 // Partition of the caller's workspace (byte offsets, each 256-byte aligned).
 struct Workspace {

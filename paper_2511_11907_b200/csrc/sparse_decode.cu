@@ -435,8 +435,9 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   // promised that q and the selection are settled: then only this kernel's writes (the partials,
   // which the previous launch's combine may still be reading) have to wait for it.
   const bool settled = (p.flags & KVSWAP_INPUTS_SETTLED) != 0;
+  const bool wait_early = settled && (p.flags & kFlagWaitEarly) != 0;
   if (!settled) pdl_wait();
-  pdl_trigger();
+  if (!wait_early) pdl_trigger();
 
   // The virtual token list is laid out for M selected groups, whatever n_selected says (slots of
   // groups beyond n_selected are simply absent), so that the split of the list does not wait for a
@@ -511,6 +512,10 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
     for (int k = 0; k < kMaxDepth; ++k)
       if (k < depth) fill(k, j0[k], warp + kWarps * k);
   }
+  if (wait_early) {                                // the first fills are in flight
+    pdl_wait();
+    pdl_trigger();
+  }
 
   Engine eng;
   eng.init(q + (int64_t(b) * p.Hq + h0) * D, lane);
@@ -542,7 +547,7 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   float* sm_acc = sm_l + kWarps * 8;                                // [kWarps][RH][D]
   eng.store(sm_m + warp * 8, sm_l + warp * 8, sm_acc + warp * RH * D);
   __syncthreads();
-  if (settled) pdl_wait();
+  if (settled && !wait_early) pdl_wait();
   for (int i = threadIdx.x; i < RH * D; i += kThreads) {
     const int hh = i / D, c = i % D;
     float mx = -INFINITY;

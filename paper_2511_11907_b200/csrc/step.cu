@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "api_internal.cuh"
+#include "combine.cuh"
 #include "common.cuh"
 
 using namespace kvswap;
@@ -195,6 +196,7 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
     // that layer's scorer finds them in the workspace and goes straight to its tiles.  The workspace
     // has two query buffers: the scorer of layer l + 1 may still be reading its own.
     const bool ahead = query_ahead_supported(p);
+    const bool merges = select_merges_with_combine(p) && (p.d == 64 || p.d == 128) && w.splits <= kMaxSplits;
     int formed_for = -1;                            // the layer whose queries the last merged launch formed
     auto score = [&](int l) -> int {
       if (probed(l)) ev(probe_opt->ev_begin);
@@ -220,14 +222,21 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
       const int32_t* nsel_l = n_selected + size_t(l) * nsel_elems;
       const bool next = l + 1 < L;
       // (the last layer's attention follows its own TopK directly: that selection is not settled)
-      const Problem& pa = next ? p_settled : p;
+      // Where the merged launch follows, the gather waits for the scorer before it as soon as its
+      // first fills are out and lets that launch start only then: its TopK, whose inputs that scorer
+      // wrote, need not wait for the gather.
+      Problem p_early = p_settled;
+      p_early.flags |= kFlagWaitEarly;
+      const Problem& pa = !next ? p : merges ? p_early : p_settled;
       if (launch_sparse_decode(pa, w, ql, layers->K[l], layers->V[l], idx_l, nsel_l, partial, out_l, lse_l,
                                static_cast<uint32_t*>(ws), stream, /*combine=*/false) != cudaSuccess)
         return KVSWAP_ERR_CUDA;
       cudaError_t e = cudaSuccess;
       const bool form = ahead && l + 2 < L;
       const void* q_ahead = form ? static_cast<const char*>(q) + size_t(l + 2) * q_bytes : nullptr;
-      const bool merged = next && select_with_combine_launch(p_settled, w, group_idx + size_t(l + 1) * idx_elems,
+      Problem p_two_back = p_settled;
+      p_two_back.flags |= kFlagInputsTwoBack;
+      const bool merged = next && select_with_combine_launch(merges ? p_two_back : p_settled, w, group_idx + size_t(l + 1) * idx_elems,
                                                              n_selected + size_t(l + 1) * nsel_elems, ws, partial, out_l,
                                                              lse_l, w.splits, p.B * p.Hq, p.d, stream, &e, q_ahead,
                                                              form ? layers->proj[l + 2] : nullptr, (l + 2) & 1);

@@ -93,7 +93,7 @@ __device__ __forceinline__ void topk_parts_body(const Problem& p, const float* _
   const int tid = threadIdx.x;
   reinterpret_cast<int4*>(hist)[tid] = make_int4(0, 0, 0, 0);
   if (tid == 0) { sh_bin = 0; sh_want = 1; sh_cnt = 0; sh_few = 0; }
-  pdl_wait();
+  if ((p.flags & kFlagInputsTwoBack) == 0) pdl_wait();
   pdl_trigger();
   const float* R = scores + int64_t(prob) * p.score_pitch;
   int32_t* out = group_idx + int64_t(prob) * p.M;
@@ -103,7 +103,8 @@ __device__ __forceinline__ void topk_parts_body(const Problem& p, const float* _
   const int base = kBins - 4 * (tid + 1);
   uint2* H = reinterpret_cast<uint2*>(top_hist + int64_t(prob) * (kKeyTopBins / 2) + base / 2);
   uint32_t* ticket = top_hist + int64_t(n_probs) * (kKeyTopBins / 2) + prob;
-  const uint2 h = *H;
+  // (loads that bypass L1: with kFlagInputsTwoBack the CTA has passed no dependency wait of its own)
+  const uint2 h = __ldcg(H);
   uint32_t key[P][4];
   const bool vec = (p.score_pitch & 3) == 0;   // rows start 16-byte aligned and are padded to whole vectors
 #pragma unroll
@@ -111,12 +112,12 @@ __device__ __forceinline__ void topk_parts_body(const Problem& p, const float* _
     const int i = q * kPartKeys + 4 * tid;
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
     if (vec) {
-      if (i < NG) x = *reinterpret_cast<const float4*>(R + i);
+      if (i < NG) x = __ldcg(reinterpret_cast<const float4*>(R + i));
     } else {
-      if (i < NG) x.x = R[i];
-      if (i + 1 < NG) x.y = R[i + 1];
-      if (i + 2 < NG) x.z = R[i + 2];
-      if (i + 3 < NG) x.w = R[i + 3];
+      if (i < NG) x.x = __ldcg(R + i);
+      if (i + 1 < NG) x.y = __ldcg(R + i + 1);
+      if (i + 2 < NG) x.z = __ldcg(R + i + 2);
+      if (i + 3 < NG) x.w = __ldcg(R + i + 3);
     }
     key[q][0] = (i < NG) ? fast_key(x.x) : 0u;
     key[q][1] = (i + 1 < NG) ? fast_key(x.y) : 0u;
