@@ -40,10 +40,10 @@ METRIC = "decode_steps_per_sec"
 UNIT = "steps/s"
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the split-K sparse-decode
-# kernel from one ncu capture at the workload's full shapes on one layer (the traffic of a launch
+# kernel from one ncu capture at the workload's full shapes on three layers (the traffic of a launch
 # does not depend on the layer count).  None for workloads that were not captured, or whose kernel
 # has changed since.  Key: (config, metadata layout, scope).
-NCU_TRAFFIC = {(5, "joint", "kv_head"): 134455808 + 3698688, (5, "per_head", "kv_head"): 134455808 + 3698688}
+NCU_TRAFFIC = {(5, "joint", "kv_head"): 134448384 + 3778816, (5, "per_head", "kv_head"): 134448384 + 3778816}
 
 
 def esz_of(dtype: int) -> int:
