@@ -160,9 +160,10 @@ int kvswap_read_device_status(const void* ws, void* cuda_stream);
  * K: [B, H_kv, N, d] kv_dtype.  proj: [H_kv, d, r] fp32, dense.  meta_out: [B, H_m, N, r]
  * meta_dtype; fp32 accumulation, one round-to-nearest-even into meta_dtype.  Rows outside
  * [n_begin, n_end) are not touched.  Requires 0 <= n_begin <= n_end <= N (empty range: no-op).
- * `ws` may be NULL here.  With a workspace of at least kvswap_workspace_bytes(shape) the bf16,
- * d = 128, r = 32 case runs on the tcgen05 tensor cores (it keeps a pre-split copy of the adapter in
- * the workspace); without one, and for every other shape, a warp-level kernel computes the same result.
+ * `ws` may be NULL here.  With a workspace of at least kvswap_workspace_bytes(shape), bf16 K with
+ * d in {64, 128} and r in {16, 32, 64} runs on the tcgen05 tensor cores (it keeps a pre-split copy of
+ * the adapter in the workspace); without one, and for every other shape, a warp-level kernel computes
+ * the same result.
  */
 int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* proj,
                         void* meta_out, int32_t n_begin, int32_t n_end,

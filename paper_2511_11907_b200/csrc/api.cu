@@ -259,8 +259,8 @@ int kvswap_project_keys(const kvswap_shape* shape, const void* K, const float* p
   if (misaligned(K) || misaligned(proj) || misaligned(meta_out)) return KVSWAP_ERR_ALIGN;
   if (n_begin < 0 || n_end < n_begin || n_end > p.N) return KVSWAP_ERR_SHAPE;
   if (n_begin == n_end) return KVSWAP_OK;
-  // The workspace is optional here: with one of at least kvswap_workspace_bytes() the bf16 / r = 32 /
-  // d = 128 case runs on tcgen05 (it needs room for the split adapter), otherwise on the warp-level path.
+  // The workspace is optional here: with one of at least kvswap_workspace_bytes() bf16 K with d in {64, 128}
+  // and r in {16, 32, 64} runs on tcgen05 (it needs room for the split adapter), otherwise on the warp-level path.
   void* scratch = nullptr;
   uint32_t* err = nullptr;
   if (ws != nullptr && !misaligned(ws)) {

@@ -1,24 +1,25 @@
 // K1 on the 5th-generation tensor cores: metadata build K_lr = Flatten(K) A (Sec. 4.2) with
 // tcgen05.mma, accumulators in tensor memory and operands staged by TMA.
 //
-// Covers bf16 K with d = 128 and r = 32 (the benchmark shapes); project_keys.cu keeps the
-// warp-level path for everything else.
+// Covers bf16 K with d in {64, 128} and r in {16, 32, 64} (r = 32, d = 128 are the benchmark
+// shapes); project_keys.cu keeps the warp-level path for everything else.
 //
 // The adapter stays fp32-exact: every entry is split into three bf16 pieces, laid out by a small
 // preparation kernel as a K-major [3r x d] operand per KV head, so one instruction shape
-// M = 128 tokens, N = 96 = 3 x 32 columns, K = 16 channels yields the three partial products side
-// by side; the epilogue adds them in fp32.  The tensor core adds into its accumulator with
-// truncation, so a chain inside tensor memory covers one KV head (8 instructions); the sum over
-// the heads of a joint row is kept in registers with round-to-nearest adds.
+// M = 128 tokens, N = 3r (48, 96 or 192) columns, K = 16 channels yields the three partial products
+// side by side; the epilogue adds them in fp32.  The tensor core adds into its accumulator with
+// truncation, so a chain inside tensor memory covers one KV head (d / 16 instructions); the sum
+// over the heads of a joint row is kept in registers with round-to-nearest adds.
 //
 // CTA = 6 warps, persistent (one per SM):
-//   warp 0   producer: per (token tile, KV head) two TMA boxes of K (128 rows x 64 channels,
-//            128-byte swizzle) and two of the split adapter into a ring of stages;
+//   warp 0   producer: per (token tile, KV head) d / 64 TMA boxes of K (128 rows x 64 channels,
+//            128-byte swizzle) and as many of the split adapter into a ring of stages;
 //   warp 1   issues the MMAs (one thread), owns the tensor-memory allocation (two accumulators);
 //   warps 2-5 epilogue: tcgen05.ld of the finished accumulator (one token row per thread), sum of
 //            the three pieces, running sum over heads, one rounding into the metadata type.
 // Stages and accumulators are handed over through mbarriers; every wait is bounded.
 #include <algorithm>
+#include <type_traits>
 
 #include "async_copy.cuh"
 #include "common.cuh"
@@ -27,19 +28,33 @@
 namespace kvswap {
 namespace {
 
-constexpr int kD = 128, kR = 32, kNcols = 3 * kR;          // channels, rank, accumulator columns
 constexpr int kTileM = 128;                                // tokens per tile
-constexpr int kStages = 3;
 constexpr uint32_t kAHalf = kTileM * 128;                  // 128 rows x 128 bytes (64 bf16 channels)
-constexpr uint32_t kBHalf = kNcols * 128;
-constexpr uint32_t kStageBytes = 2 * kAHalf + 2 * kBHalf;  // 57344
 constexpr int kThreadsUmma = 6 * 32;
-constexpr uint32_t kTmemCols = 256;                        // two accumulators of 96 columns, at 0 and 128
+constexpr size_t kMaxDynamicSmem = 227 * 1024;
+
+// Sizes for head dimension D and rank R.
+template <int D, int R>
+struct Cfg {
+  static constexpr int kD = D, kR = R;
+  static constexpr int kNcols = 3 * R;                                   // accumulator columns: the three pieces side by side
+  static constexpr int kHalves = D / 64;                                 // 128-byte-wide boxes per operand row
+  static constexpr uint32_t kBHalf = uint32_t(kNcols) * 128;
+  static constexpr uint32_t kStageBytes = kHalves * (kAHalf + kBHalf);   // d = 128, r = 32: 57344
+  static constexpr int kStages = (3 * size_t(kStageBytes) + 1024 <= kMaxDynamicSmem) ? 3 : 2;
+  static constexpr uint32_t kAccStride = (kNcols <= 128) ? 128 : 256;    // tensor-memory columns between the two accumulators
+  static constexpr uint32_t kTmemCols = 2 * kAccStride;
+  static_assert((D == 64 || D == 128) && (R == 16 || R == 32 || R == 64), "shapes of the tcgen05 projection");
+  static_assert(kNcols % 16 == 0 && kNcols <= 256, "N of a 128-row tcgen05.mma");
+};
+constexpr int kMaxStages = 3;
 
 // ---- the adapter as three bf16 pieces, [g][piece * r + j][c] (K-major rows of d channels) ----------
-__global__ void split_adapter_kernel(const float* __restrict__ proj, __nv_bfloat16* __restrict__ bsplit, int n) {
+__global__ void split_adapter_kernel(const float* __restrict__ proj, __nv_bfloat16* __restrict__ bsplit, int n, int kD,
+                                     int kR) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;     // over [g][c][j]
   if (i >= n) return;
+  const int kNcols = 3 * kR;
   const int j = i % kR, c = (i / kR) % kD, g = i / (kR * kD);
   const float v = proj[i];
   const __nv_bfloat16 hi = __float2bfloat16_rn(v);
@@ -78,24 +93,43 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[32]) { tmem_ld32(taddr, v); }
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[16]) { tmem_ld16(taddr, v); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 struct UmmaShared {
-  unsigned long long full[kStages];        // stage loaded (TMA bytes)
-  unsigned long long empty[kStages];       // stage consumed (MMA commit)
+  unsigned long long full[kMaxStages];     // stage loaded (TMA bytes)
+  unsigned long long empty[kMaxStages];    // stage consumed (MMA commit)
   unsigned long long acc_full[2];          // accumulator finished (MMA commit)
   unsigned long long acc_empty[2];         // accumulator read out (4 epilogue warps)
   uint32_t tmem_base;
   uint32_t abort;
 };
 
-template <typename META_T>
+// D = channels multiplied per stage.  PAIR (D = 128 with heads of 64 channels, joint metadata): a stage
+// holds two KV heads, one per 64-channel half, so the chain inside tensor memory sums a pair of heads
+// and there are half as many stages to hand over.
+template <int D, int R, typename META_T, bool PAIR>
 __global__ void __launch_bounds__(kThreadsUmma, 1)
 project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_b,
                          META_T* __restrict__ meta, int n_begin, int n_end, int tiles_per_row,
                          uint32_t* __restrict__ err) {
+  using C = Cfg<D, R>;
+  constexpr int kD = D, kR = R, kNcols = C::kNcols, kStages = C::kStages, kHalves = C::kHalves;
+  constexpr uint32_t kBHalf = C::kBHalf, kStageBytes = C::kStageBytes, kTmemCols = C::kTmemCols, kAccStride = C::kAccStride;
+  constexpr int kChunk = (R < 32) ? R : 32;                // accumulator columns per tensor-memory load
   extern __shared__ unsigned char dyn_raw[];
   const uint32_t stage0 = (smem_addr(dyn_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
   __shared__ UmmaShared sh;
@@ -117,7 +151,7 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
   const uint32_t tmem = sh.tmem_base;
 
   // Work: contiguous range of (sequence, metadata head, token tile) items; a step = (item, KV head).
-  const int g_count = (p.Hm == 1) ? p.Hkv : 1;
+  const int g_count = PAIR ? p.Hkv / 2 : (p.Hm == 1) ? p.Hkv : 1;      // stages per (token tile) item
   const int64_t items = int64_t(p.B) * p.Hm * tiles_per_row;
   const int64_t first = items * blockIdx.x / gridDim.x, last = items * (blockIdx.x + 1) / gridDim.x;
   const int n_steps = int(last - first) * g_count;
@@ -131,32 +165,34 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
         const int64_t item = first + s / g_count;
         const int tile = int(item % tiles_per_row), bh = int(item / tiles_per_row);
         const int hm = bh % p.Hm, b = bh / p.Hm;
-        const int g = ((p.Hm == 1) ? 0 : hm) + s % g_count;
+        const int g = ((p.Hm == 1) ? 0 : hm) + (s % g_count) * (PAIR ? 2 : 1);
         const uint32_t dst = stage0 + uint32_t(stage) * kStageBytes, bar = smem_addr(&sh.full[stage]);
         mbar_arrive_expect_tx(bar, kStageBytes);
         const int n0 = n_begin + tile * kTileM;
-        tma_load_4d(dst, &map_k, bar, 0, n0, g, b);
-        tma_load_4d(dst + kAHalf, &map_k, bar, 64, n0, g, b);
-        tma_load_2d(dst + 2 * kAHalf, &map_b, bar, 0, g * kNcols);
-        tma_load_2d(dst + 2 * kAHalf + kBHalf, &map_b, bar, 64, g * kNcols);
+#pragma unroll
+        for (int h = 0; h < kHalves; ++h) {
+          const int c0 = PAIR ? 0 : 64 * h, gh = PAIR ? g + h : g;       // channels and head of this half
+          tma_load_4d(dst + uint32_t(h) * kAHalf, &map_k, bar, c0, n0, gh, b);
+          tma_load_2d(dst + kHalves * kAHalf + uint32_t(h) * kBHalf, &map_b, bar, c0, gh * kNcols);
+        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ================================ MMA issuer ============================================
     if (lane == 0) {
-      // M = 128, N = 96, fp32 accumulate, bf16 x bf16, both operands K-major
+      // M = 128, N = 3r, fp32 accumulate, bf16 x bf16, both operands K-major
       constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(kNcols >> 3) << 17) | (uint32_t(kTileM >> 4) << 24);
       for (int s = 0; s < n_steps; ++s) {
         const int stage = s % kStages, use = s / kStages, buf = s & 1, acc_use = s >> 1;
         if (acc_use > 0 && !mbar_wait(smem_addr(&sh.acc_empty[buf]), uint32_t(acc_use - 1) & 1u)) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutEmpty); break; }
         if (!mbar_wait(smem_addr(&sh.full[stage]), uint32_t(use) & 1u)) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutFull); break; }
         tc_fence_after();
-        const uint32_t a0 = stage0 + uint32_t(stage) * kStageBytes, b0 = a0 + 2 * kAHalf;
+        const uint32_t a0 = stage0 + uint32_t(stage) * kStageBytes, b0 = a0 + kHalves * kAHalf;
 #pragma unroll
         for (int k = 0; k < kD / 16; ++k) {
           const uint32_t half = k >> 2, koff = uint32_t(k & 3) * 32u;     // 16 channels = 32 bytes inside the swizzle row
-          umma_bf16(tmem + uint32_t(buf) * 128u, umma_desc(a0 + half * kAHalf + koff), umma_desc(b0 + half * kBHalf + koff),
+          umma_bf16(tmem + uint32_t(buf) * kAccStride, umma_desc(a0 + half * kAHalf + koff), umma_desc(b0 + half * kBHalf + koff),
                     idesc, k > 0 ? 1u : 0u);
         }
         umma_commit(smem_addr(&sh.empty[stage]));         // the stage may be refilled once these MMAs have read it
@@ -177,17 +213,20 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
       ok = __all_sync(0xffffffffu, mbar_wait(smem_addr(&sh.acc_full[buf]), uint32_t(acc_use) & 1u));
       if (!ok) { if (lane == 0) { sh.abort = 1; if (err) atomicExch(err, kDevTimeoutFull); } break; }
       tc_fence_after();
-      const uint32_t taddr = tmem + (uint32_t(quarter * 32) << 16) + uint32_t(buf) * 128u;
-      float hi[32], mid[32], lo[32];
-      tmem_ld32(taddr, hi);
-      tmem_ld32(taddr + 32, mid);
-      tmem_ld32(taddr + 64, lo);
-      tmem_ld_wait();
+      const uint32_t taddr = tmem + (uint32_t(quarter * 32) << 16) + uint32_t(buf) * kAccStride;
+#pragma unroll
+      for (int c0 = 0; c0 < kR; c0 += kChunk) {            // the pieces of columns c0 .. c0 + kChunk - 1 sit kR columns apart
+        float hi[kChunk], mid[kChunk], lo[kChunk];
+        tmem_ld_cols(taddr + c0, hi);
+        tmem_ld_cols(taddr + kR + c0, mid);
+        tmem_ld_cols(taddr + 2 * kR + c0, lo);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < kChunk; ++j) acc[c0 + j] += (lo[j] + mid[j]) + hi[j];
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_addr(&sh.acc_empty[buf]));
-#pragma unroll
-      for (int j = 0; j < kR; ++j) acc[j] += (lo[j] + mid[j]) + hi[j];
       if ((s + 1) % g_count == 0) {                        // last head of the item: one rounding, one row out
         const int64_t item = first + s / g_count;
         const int tile = int(item % tiles_per_row), bh = int(item / tiles_per_row);
@@ -205,6 +244,7 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
 #pragma unroll
             for (int j = 0; j < kR / 16; ++j)
               reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            static_assert(kR % 16 == 0, "whole 16-byte vectors per row");
           } else if constexpr (sizeof(META_T) == 2) {
             uint32_t w[kR / 2];
 #pragma unroll
@@ -243,46 +283,80 @@ project_keys_umma_kernel(Problem p, const __grid_constant__ CUtensorMap map_k, c
 
 }  // namespace
 
-size_t project_keys_umma_scratch_bytes(const Problem& p) {
-  if (p.kv_dtype != KVSWAP_BF16 || p.d != kD || p.r != kR) return 0;
-  return size_t(p.Hkv) * kNcols * kD * sizeof(__nv_bfloat16);
+static bool umma_shape(const Problem& p) {
+  return p.kv_dtype == KVSWAP_BF16 && (p.d == 64 || p.d == 128) && (p.r == 16 || p.r == 32 || p.r == 64);
 }
 
-// Returns true (and sets *result) when this path took the problem.
-bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
-                                  int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result) {
-  if (scratch == nullptr || project_keys_umma_scratch_bytes(p) == 0) return false;
-  if (p.kv_sn != kD && (p.kv_sn * 2) % 16 != 0) return false;
-  EncodeTiledFn enc = tensor_map_encoder();
-  if (enc == nullptr) return false;
-  CUtensorMap map_k, map_b;
-  if (!make_rows_tensor_map(&map_k, K, 2, true, kD, p.N, p.Hkv, p.B, p.kv_sn, p.kv_sh, p.kv_sb, kTileM)) return false;
-  {
-    const cuuint64_t dims[2] = {cuuint64_t(kD), cuuint64_t(p.Hkv) * kNcols};
-    const cuuint64_t strides[1] = {cuuint64_t(kD) * 2};
-    const cuuint32_t box[2] = {64, kNcols}, estr[2] = {1, 1};
-    if (enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, scratch, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return false;
-  }
-  const int n_proj = p.Hkv * kD * kR;
-  split_adapter_kernel<<<(n_proj + 255) / 256, 256, 0, st>>>(proj, static_cast<__nv_bfloat16*>(scratch), n_proj);
-  *result = cudaGetLastError();
-  if (*result != cudaSuccess) return true;
+size_t project_keys_umma_scratch_bytes(const Problem& p) {
+  if (!umma_shape(p)) return 0;
+  return size_t(p.Hkv) * 3 * p.r * p.d * sizeof(__nv_bfloat16);
+}
 
+namespace {
+
+template <int D, int R, bool PAIR>
+cudaError_t launch_umma(const Problem& p, const CUtensorMap& map_k, const CUtensorMap& map_b, void* meta, int n_begin,
+                        int n_end, uint32_t* err, cudaStream_t st) {
+  using C = Cfg<D, R>;
   const int tiles_per_row = (n_end - n_begin + kTileM - 1) / kTileM;
   const int64_t items = int64_t(p.B) * p.Hm * tiles_per_row;
   const int ctas = int(std::max<int64_t>(1, std::min<int64_t>(kNumSMs, items)));
-  const size_t smem = size_t(kStages) * kStageBytes + 1024;
+  const size_t smem = size_t(C::kStages) * C::kStageBytes + 1024;
   auto go = [&](auto kern, auto* meta_t) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
     kern<<<ctas, kThreadsUmma, smem, st>>>(p, map_k, map_b, meta_t, n_begin, n_end, tiles_per_row, err);
     return cudaGetLastError();
   };
-  if (p.meta_dtype == KVSWAP_E4M3) *result = go(project_keys_umma_kernel<e4m3_t>, static_cast<e4m3_t*>(meta));
-  else if (p.meta_dtype == KVSWAP_F16) *result = go(project_keys_umma_kernel<__half>, static_cast<__half*>(meta));
-  else *result = go(project_keys_umma_kernel<float>, static_cast<float*>(meta));
+  if constexpr (R == 32) {                                 // 8-bit metadata exists for r = 32 only
+    if (p.meta_dtype == KVSWAP_E4M3) return go(project_keys_umma_kernel<D, R, e4m3_t, PAIR>, static_cast<e4m3_t*>(meta));
+  }
+  if (p.meta_dtype == KVSWAP_E4M3) return cudaErrorInvalidValue;
+  if (p.meta_dtype == KVSWAP_F16) return go(project_keys_umma_kernel<D, R, __half, PAIR>, static_cast<__half*>(meta));
+  return go(project_keys_umma_kernel<D, R, float, PAIR>, static_cast<float*>(meta));
+}
+
+}  // namespace
+
+// Returns true (and sets *result) when this path took the problem.
+bool try_launch_project_keys_umma(const Problem& p, const void* K, const float* proj, void* meta, int n_begin,
+                                  int n_end, void* scratch, uint32_t* err, cudaStream_t st, cudaError_t* result) {
+  if (scratch == nullptr || project_keys_umma_scratch_bytes(p) == 0) return false;
+  if (p.meta_dtype == KVSWAP_E4M3 && p.r != 32) return false;
+  // Heads of 64 channels are multiplied in pairs where one metadata row sums all heads; alone they
+  // leave each stage half as much to do, and at r = 16 the warp-level kernel is the faster one.
+  const bool pair = p.d == 64 && p.Hm == 1 && p.Hkv % 2 == 0;
+  if (p.d == 64 && !pair && p.r == 16) return false;
+  if (p.kv_sn != p.d && (p.kv_sn * 2) % 16 != 0) return false;
+  EncodeTiledFn enc = tensor_map_encoder();
+  if (enc == nullptr) return false;
+  const int ncols = 3 * p.r;
+  CUtensorMap map_k, map_b;
+  if (!make_rows_tensor_map(&map_k, K, 2, true, p.d, p.N, p.Hkv, p.B, p.kv_sn, p.kv_sh, p.kv_sb, kTileM)) return false;
+  {
+    const cuuint64_t dims[2] = {cuuint64_t(p.d), cuuint64_t(p.Hkv) * ncols};
+    const cuuint64_t strides[1] = {cuuint64_t(p.d) * 2};
+    const cuuint32_t box[2] = {64, cuuint32_t(ncols)}, estr[2] = {1, 1};
+    if (enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, scratch, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  const int n_proj = p.Hkv * p.d * p.r;
+  split_adapter_kernel<<<(n_proj + 255) / 256, 256, 0, st>>>(proj, static_cast<__nv_bfloat16*>(scratch), n_proj, p.d, p.r);
+  *result = cudaGetLastError();
+  if (*result != cudaSuccess) return true;
+  auto by_rank = [&](auto d_tag, auto pair_tag) {
+    constexpr int D = decltype(d_tag)::value;
+    constexpr bool P = decltype(pair_tag)::value;
+    return p.r == 16   ? launch_umma<D, 16, P>(p, map_k, map_b, meta, n_begin, n_end, err, st)
+           : p.r == 32 ? launch_umma<D, 32, P>(p, map_k, map_b, meta, n_begin, n_end, err, st)
+                       : launch_umma<D, 64, P>(p, map_k, map_b, meta, n_begin, n_end, err, st);
+  };
+  using D128 = std::integral_constant<int, 128>;
+  using D64 = std::integral_constant<int, 64>;
+  *result = pair         ? by_rank(D128(), std::true_type())
+            : p.d == 128 ? by_rank(D128(), std::false_type())
+                         : by_rank(D64(), std::false_type());
   return true;
 }
 

@@ -363,6 +363,34 @@ def test_project_keys_without_workspace_takes_the_warp_level_path():
         assert np.mean(got != meta_or.astype(np.float32)) < 0.02
 
 
+@pytest.mark.parametrize("head_dim,rank", [(64, 16), (64, 32), (64, 64), (128, 16), (128, 64)])
+@pytest.mark.parametrize("meta_heads", [1, "per_head"])
+def test_project_keys_tensor_core_shapes(head_dim, rank, meta_heads):
+    """bf16 K with d in {64, 128} and r in {16, 32, 64}: with a workspace the projection runs on
+    tcgen05 (instruction width 3r = 48, 96 or 192 columns, d / 64 boxes per operand row), without one on
+    the warp-level kernel; both against the oracle, over 9 token tiles with a ragged last one and
+    over a token range that starts and ends inside a tile."""
+    wl = small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=head_dim, rank=rank, group_size=8,
+               n_ctx=1024 + 77, n_q_heads=8, n_kv_heads=4, batch=2)
+    mh = 1 if meta_heads == 1 else wl.n_kv_heads
+    li = W.make_layer(wl, 0, mh)
+    dl = DeviceLayer(li, KV)
+    meta_or = O.project_keys(li.K, li.proj, mh, "f16")
+    tol = project_tolerance(li.K, li.proj, mh, meta_or, wl.meta_dtype)
+    for ws in (dl.ws, None):
+        dl.meta.fill_(float("nan"))
+        kv.kvswap_project_keys(dl.shape, dl.K, dl.proj, dl.meta, 0, wl.n_ctx, ws)
+        torch.cuda.synchronize()
+        got = rt.to_host_f32(dl.meta)
+        assert np.all(np.abs(got.astype(np.float64) - meta_or.astype(np.float64)) <= tol)
+        assert np.mean(got != meta_or.astype(np.float32)) < 0.02
+    dl.meta.fill_(123.0)
+    got = dl.project(n_begin=130, n_end=130 + 517)
+    assert np.all(got[:, :, :130] == 123.0) and np.all(got[:, :, 647:] == 123.0)
+    assert np.all(np.abs(got[:, :, 130:647].astype(np.float64) - meta_or[:, :, 130:647].astype(np.float64)) <= tol[:, :, 130:647])
+    assert kv.kvswap_read_device_status(dl.ws) == 0
+
+
 def test_strided_kv_and_metadata_views():
     """K and V interleaved in one buffer (row stride 2d) and metadata rows padded."""
     wl = small(kv_dtype=W.BF16, q_dtype=W.BF16, meta_dtype=W.F16, head_dim=128, rank=32, n_ctx=517, group_size=8)
