@@ -316,7 +316,8 @@ def call_rooflines(torch, kv, wl, dw, meta, shape, idx, nsel, out, ws, layers_us
               "as a CUDA graph (no host in the loop); every call waits for the kernel before it")
     roof = {"bound": "hbm", "kernel": "kvswap_sparse_decode (gather split-K + combine)",
             "achieved": gbs(decode_bytes, dec_wait_us), "peak": peak, "unit": "GB/s",
-            "frac": gbs(decode_bytes, dec_wait_us) / peak, "peak_kind": peak_kind, "traffic": traffic,
+            "frac": gbs(decode_bytes, dec_wait_us) / peak, "frac_waiting_for_previous_kernel": gbs(decode_bytes, dec_wait_us) / peak,
+            "peak_kind": peak_kind, "traffic": traffic,
             "algorithmic_bytes_per_launch": decode_bytes, "avg_ms": dec_wait_us / 1e3, "launches_timed": dec_calls,
             "timing": timing,
             "avg_ms_inputs_settled": dec_settled_us / 1e3, "frac_inputs_settled": gbs(decode_bytes, dec_settled_us) / peak,
@@ -538,6 +539,7 @@ def run_ours(args, wl):
                                                                           nsel[l], None, ws)) for l in range(L)], 400)
     _, select_bytes = workload_bytes(wl, meta_heads, S)
     fp8 = fp8_metadata_leg(torch, kv, rt, wl, dw, meta_heads, scope, idx, nsel, dev, peak) if wl.meta_dtype == W.F16 and wl.rank == 32 else None
+    shapes = prefill_shapes_leg(torch, kv, rt, wl, dw, dev, peak) if wl.kv_dtype == W.BF16 and not args.no_secondary else None
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         cpu = cpu_baseline(wl, dw, meta_heads, args.scope, rt)
@@ -586,7 +588,8 @@ def run_ours(args, wl):
         "metadata_8bit": fp8,
         "prefill": {"project_keys_ms_all_layers": prefill_ms,
                     "keys_projected_per_sec": keys_per_step / prefill_ms * 1e3,
-                    "read_gbs": L * wl.batch * wl.n_kv_heads * wl.n_ctx * wl.head_dim * esz[wl.kv_dtype] / prefill_ms / 1e6},
+                    "read_gbs": L * wl.batch * wl.n_kv_heads * wl.n_ctx * wl.head_dim * esz[wl.kv_dtype] / prefill_ms / 1e6,
+                    "other_shapes_one_layer": shapes},
         "selection_overlap_ratio": statistics.mean(overlaps) if overlaps else None,
         "clocks": clocks,
     }
@@ -595,6 +598,41 @@ def run_ours(args, wl):
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def prefill_shapes_leg(torch, kv, rt, wl, dw, dev, peak):
+    """kvswap_project_keys (K1) on one layer of the workload's size for the other head dimensions and ranks
+    the tensor-core projection takes (bf16 K, joint adapter): with a workspace (tcgen05) and without one
+    (the warp-level kernel), read bandwidth over the K bytes.  Random adapters; timing only."""
+    res = {}
+    B, Hkv, N = wl.batch, wl.n_kv_heads, wl.n_ctx
+    for d in (128, 64):
+        K = dw.K[0] if d == wl.head_dim else (torch.randn((B, Hkv, N, d), device=dev, dtype=torch.float32) * 0.5).to(torch.bfloat16)
+        for r in (16, 32, 64):
+            shape = kv.make_shape(batch=B, n_ctx=N, n_q_heads=wl.n_q_heads, n_kv_heads=Hkv, head_dim=d, rank=r,
+                                  meta_heads=1, group_size=wl.group_size, top_k=wl.top_k, kv_dtype=W.BF16,
+                                  meta_dtype=W.F16, q_dtype=W.BF16)
+            proj = torch.randn((Hkv, d, r), device=dev, dtype=torch.float32) * 0.05
+            meta = torch.empty((B, 1, N, r), device=dev, dtype=torch.float16)
+            ws = rt.alloc_workspace(shape, dev)
+            us = []
+            for w in (ws, None):
+                for _ in range(3):
+                    kv.kvswap_project_keys(shape, K, proj, meta, 0, N, w)
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(10):
+                    kv.kvswap_project_keys(shape, K, proj, meta, 0, N, w)
+                b.record()
+                torch.cuda.synchronize()
+                us.append(a.elapsed_time(b) * 100.0)
+            nbytes = B * Hkv * N * d * 2
+            res[f"d{d}_r{r}"] = {"us": us[0], "read_gbs": nbytes / us[0] / 1e3, "frac": nbytes / us[0] / 1e3 / peak,
+                                 "us_without_workspace": us[1]}
+            del meta, ws, proj
+        del K
+    return res
 
 
 def fp8_metadata_leg(torch, kv, rt, wl, dw, meta_heads, scope, idx, nsel, dev, peak):
