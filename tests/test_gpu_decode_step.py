@@ -105,6 +105,45 @@ def test_decode_step_head_dim_64(meta_heads):
     _run_case(wl, meta_heads, W.SCOPE_KV_HEAD)
 
 
+@pytest.mark.parametrize("meta_heads", ["joint", "per_head"])
+def test_decode_steps_back_to_back_with_alternating_queries(meta_heads):
+    """Steps enqueued without a pause, alternating between two query sets: inside a step the TopK of a
+    layer does not wait for the gather before it, the scorer reads queries that the launch before it
+    formed, and consecutive steps reuse the same workspace buffers -- every step must still give what
+    the per-layer calls give for its queries."""
+    wl = W.CONFIGS[5].reduced("cfg5-soak", layers=6, batch=2, n_ctx=16384 + 5, top_k=96, calib_rows=1024, walk_steps=2)
+    dw = DW.build(wl, 1 if meta_heads == "joint" else wl.n_kv_heads, W.SCOPE_KV_HEAD, reserve_bytes=1 << 30)
+    ws = rt.alloc_workspace(dw.shape)
+    for l in range(wl.layers):
+        kv.kvswap_project_keys(dw.shape, dw.K[l], dw.proj[l], dw.meta[l], 0, wl.n_ctx, ws)
+    refs = []
+    for w in range(2):
+        out, lse, idx, nsel = _step_buffers(dw)
+        q = dw.q_walk[w]
+        for l in range(wl.layers):
+            kv.kvswap_score_select(dw.shape, q[l], dw.proj[l], dw.meta[l], idx[l], nsel[l], None, ws)
+            kv.kvswap_sparse_decode(dw.shape, q[l], dw.K[l], dw.V[l], idx[l], nsel[l], out[l], lse[l], ws)
+        refs.append((out, lse, idx, nsel))
+    torch.cuda.synchronize()
+    assert not torch.equal(refs[0][2], refs[1][2])          # the two query sets select differently
+    layers = dw.layer_tables(1)
+    bufs = [_step_buffers(dw) for _ in range(4)]
+    bad = torch.zeros((), dtype=torch.int64, device="cuda")
+    for i in range(120):
+        out, lse, idx, nsel = bufs[i % 4]
+        kv.kvswap_decode_step(dw.shape, layers, dw.q_walk[i % 2], out, lse, idx, nsel, ws)
+        if i % 4 == 3:                                       # four steps back to back, then all four are checked
+            for j in range(4):
+                got, want = bufs[j], refs[j % 2]
+                differs = torch.zeros((), dtype=torch.bool, device="cuda")
+                for g, r in zip(got, want):
+                    differs |= (g != r).any()
+                bad += differs.to(torch.int64)
+    torch.cuda.synchronize()
+    assert int(bad) == 0
+    assert kv.kvswap_read_device_status(ws) == 0
+
+
 def test_decode_step_fp32_wide_rank_per_head():
     """fp32 everywhere, rank 128 per-head metadata, batch 64 (generic kernels on both streams)."""
     wl = W.CONFIGS[1].reduced("cfg1-wide", layers=6, batch=64, n_ctx=512, rank=128, head_dim=128, n_q_heads=32,
