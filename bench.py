@@ -43,7 +43,7 @@ UNIT = "steps/s"
 # kernel from one ncu capture at the workload's full shapes on three layers (the traffic of a launch
 # does not depend on the layer count).  None for workloads that were not captured, or whose kernel
 # has changed since.  Key: (config, metadata layout, scope).
-NCU_TRAFFIC = {(5, "joint", "kv_head"): 134448384 + 3778816, (5, "per_head", "kv_head"): 134448384 + 3778816}
+NCU_TRAFFIC = {(5, "joint", "kv_head"): 134451029 + 3957163, (5, "per_head", "kv_head"): 134451029 + 3957163}
 
 
 def esz_of(dtype: int) -> int:
