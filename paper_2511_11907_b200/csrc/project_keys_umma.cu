@@ -32,6 +32,7 @@ constexpr int kTileM = 128;                                // tokens per tile
 constexpr uint32_t kAHalf = kTileM * 128;                  // 128 rows x 128 bytes (64 bf16 channels)
 constexpr int kThreadsUmma = 6 * 32;
 constexpr size_t kMaxDynamicSmem = 227 * 1024;
+constexpr int kMaxStages = 6;
 
 // Sizes for head dimension D and rank R.
 template <int D, int R>
@@ -41,13 +42,15 @@ struct Cfg {
   static constexpr int kHalves = D / 64;                                 // 128-byte-wide boxes per operand row
   static constexpr uint32_t kBHalf = uint32_t(kNcols) * 128;
   static constexpr uint32_t kStageBytes = kHalves * (kAHalf + kBHalf);   // d = 128, r = 32: 57344
-  static constexpr int kStages = (3 * size_t(kStageBytes) + 1024 <= kMaxDynamicSmem) ? 3 : 2;
+  // as many stages as fit beside the 1 KB of alignment slack, six at most (d = 128: 4 at r = 32, 5 at r = 16, 2 at r = 64)
+  static constexpr int kFit = int((kMaxDynamicSmem - 1024) / kStageBytes);
+  static constexpr int kStages = kFit > kMaxStages ? kMaxStages : kFit;
+  static_assert(kStages >= 2, "at least two stages");
   static constexpr uint32_t kAccStride = (kNcols <= 128) ? 128 : 256;    // tensor-memory columns between the two accumulators
   static constexpr uint32_t kTmemCols = 2 * kAccStride;
   static_assert((D == 64 || D == 128) && (R == 16 || R == 32 || R == 64), "shapes of the tcgen05 projection");
   static_assert(kNcols % 16 == 0 && kNcols <= 256, "N of a 128-row tcgen05.mma");
 };
-constexpr int kMaxStages = 3;
 
 // ---- the adapter as three bf16 pieces, [g][piece * r + j][c] (K-major rows of d channels) ----------
 __global__ void split_adapter_kernel(const float* __restrict__ proj, __nv_bfloat16* __restrict__ bsplit, int n, int kD,
