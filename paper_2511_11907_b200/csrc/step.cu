@@ -236,10 +236,11 @@ static int decode_step_impl(const kvswap_shape* shape, const kvswap_layers* laye
       const void* q_ahead = form ? static_cast<const char*>(q) + size_t(l + 2) * q_bytes : nullptr;
       Problem p_two_back = p_settled;
       p_two_back.flags |= kFlagInputsTwoBack;
-      const bool merged = next && select_with_combine_launch(merges ? p_two_back : p_settled, w, group_idx + size_t(l + 1) * idx_elems,
-                                                             n_selected + size_t(l + 1) * nsel_elems, ws, partial, out_l,
-                                                             lse_l, w.splits, p.B * p.Hq, p.d, stream, &e, q_ahead,
-                                                             form ? layers->proj[l + 2] : nullptr, (l + 2) & 1);
+      const bool merged = next && merges &&
+                          select_with_combine_launch(p_two_back, w, group_idx + size_t(l + 1) * idx_elems,
+                                                     n_selected + size_t(l + 1) * nsel_elems, ws, partial, out_l, lse_l,
+                                                     w.splits, p.B * p.Hq, p.d, stream, &e, q_ahead,
+                                                     form ? layers->proj[l + 2] : nullptr, (l + 2) & 1);
       if (merged && form && e == cudaSuccess) formed_for = l + 2;
       if (!merged) {
         e = launch_combine_only(p, w, partial, out_l, lse_l, stream);
