@@ -71,7 +71,7 @@ typedef enum {
   KVSWAP_ERR_WORKSPACE = 5,   /* ws_bytes smaller than kvswap_workspace_bytes()              */
   KVSWAP_ERR_UNSUPPORTED = 6, /* valid request outside the implemented range                 */
   KVSWAP_ERR_CUDA = 7,        /* a CUDA runtime call or kernel launch failed                 */
-  KVSWAP_ERR_INDEX = 8,       /* reserved: out-of-range group index seen by a checking build */
+  KVSWAP_ERR_INDEX = 8,       /* device status: a group index or count out of range was seen (KVSWAP_CHECK_INDICES) */
   KVSWAP_ERR_STATIC_SCRATCH = 9, /* problem needs more than KVSWAP_STATIC_SCRATCH_BYTES of scratch */
   KVSWAP_ERR_TIMEOUT = 10     /* a kernel gave up a bounded wait; its outputs are invalid     */
 } kvswap_status;
@@ -108,8 +108,13 @@ typedef enum { KVSWAP_SCOPE_KV_HEAD = 0, KVSWAP_SCOPE_ALL_HEADS = 1 } kvswap_sco
  *       448 and the bulk of the values above 2^-6 (e = 0 suits keys of unit scale).  Supported for
  *       r = 32, G a power of two <= 32 and dense metadata rows (else KVSWAP_ERR_UNSUPPORTED); not with
  *       KVSWAP_SCORE_SOFTMAX.
+ *   KVSWAP_CHECK_INDICES   a debugging aid for callers that build their own index lists: besides
+ *       skipping them, kvswap_sparse_decode (and the steps built on it) records in the device
+ *       status word of `ws` that it met a group index outside [0, NG) other than the padding
+ *       value -1, or an n_selected outside [0, M]; kvswap_read_device_status then returns
+ *       KVSWAP_ERR_INDEX.  Results are those without the flag.
  */
-enum { KVSWAP_INPUTS_SETTLED = 1, KVSWAP_SCORE_SOFTMAX = 2 };
+enum { KVSWAP_INPUTS_SETTLED = 1, KVSWAP_SCORE_SOFTMAX = 2, KVSWAP_CHECK_INDICES = 4 };
 #define KVSWAP_META_EXP(e) ((int32_t)(((uint32_t)(e) & 0xffu) << 8))
 
 /*
@@ -147,7 +152,9 @@ int kvswap_validate_shape(const kvswap_shape* shape);
  *                             above); a workspace that was never cleared selects wrong groups.
  *   kvswap_read_device_status waits for `cuda_stream` to drain (the only call of the library that
  *                             synchronises), then returns KVSWAP_OK, or KVSWAP_ERR_TIMEOUT if a
- *                             kernel using `ws` has given up a wait since the word was cleared.
+ *                             kernel using `ws` has given up a wait since the word was cleared,
+ *                             or KVSWAP_ERR_INDEX if a call with KVSWAP_CHECK_INDICES has met an
+ *                             index out of range since then.
  */
 int kvswap_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);
 int kvswap_read_device_status(const void* ws, void* cuda_stream);

@@ -18,6 +18,7 @@ KVSWAP_F32, KVSWAP_BF16, KVSWAP_F16, KVSWAP_E4M3 = 0, 1, 2, 3
 KVSWAP_SCOPE_KV_HEAD, KVSWAP_SCOPE_ALL_HEADS = 0, 1
 KVSWAP_INPUTS_SETTLED = 1      # kvswap_shape.flags
 KVSWAP_SCORE_SOFTMAX = 2
+KVSWAP_CHECK_INDICES = 4
 
 
 def KVSWAP_META_EXP(e: int) -> int:
@@ -210,7 +211,8 @@ def kvswap_read_probe(buf, n_bytes: int, sink=None, stream=None) -> None:
 
 
 def kvswap_read_device_status(ws, stream=None) -> int:
-    """Synchronises the stream; returns 0, or KVSWAP_ERR_TIMEOUT (10) if a kernel gave up a wait."""
+    """Synchronises the stream; returns 0, KVSWAP_ERR_TIMEOUT (10) if a kernel gave up a wait, or
+    KVSWAP_ERR_INDEX (8) if a call with KVSWAP_CHECK_INDICES met an index out of range."""
     return int(load().kvswap_read_device_status(_ptr(ws), _stream(stream)))
 
 

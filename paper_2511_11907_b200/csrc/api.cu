@@ -4,6 +4,7 @@
 #include <algorithm>
 
 #include "api_internal.cuh"
+#include "async_copy.cuh"
 #include "common.cuh"
 #include "topk_keys.cuh"
 
@@ -28,7 +29,8 @@ int resolve(const kvswap_shape* s, Problem* p) {
   if (s->n_q_heads % s->n_kv_heads != 0) return KVSWAP_ERR_SHAPE;
   if (s->meta_heads != 1 && s->meta_heads != s->n_kv_heads) return KVSWAP_ERR_SHAPE;
   if (s->scope != KVSWAP_SCOPE_KV_HEAD && s->scope != KVSWAP_SCOPE_ALL_HEADS) return KVSWAP_ERR_SHAPE;
-  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED | KVSWAP_SCORE_SOFTMAX | 0xff00)) != 0) return KVSWAP_ERR_SHAPE;
+  if ((s->flags & ~int32_t(KVSWAP_INPUTS_SETTLED | KVSWAP_SCORE_SOFTMAX | KVSWAP_CHECK_INDICES | 0xff00)) != 0)
+    return KVSWAP_ERR_SHAPE;
   const int meta_exp = int(int8_t((s->flags >> 8) & 0xff));
   if (meta_exp < -64 || meta_exp > 63 || (meta_exp != 0 && s->meta_dtype != KVSWAP_E4M3)) return KVSWAP_ERR_SHAPE;
   if (s->n_ctx > (1 << 30) || s->batch > 65535 || s->n_q_heads > 4096) return KVSWAP_ERR_SHAPE;
@@ -399,7 +401,7 @@ int kvswap_read_device_status(const void* ws, void* cuda_stream) {
   uint32_t word = 0;
   if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
   if (cudaStreamSynchronize(stream) != cudaSuccess) return KVSWAP_ERR_CUDA;
-  return word == 0 ? KVSWAP_OK : KVSWAP_ERR_TIMEOUT;
+  return word == kDevOk ? KVSWAP_OK : word == kDevBadIndex ? KVSWAP_ERR_INDEX : KVSWAP_ERR_TIMEOUT;
 }
 
 const char* kvswap_status_string(int status) {

@@ -19,6 +19,7 @@ enum : uint32_t {
   kDevOk = 0,
   kDevTimeoutFull = 1,    // a consumer waited for staged data that never arrived
   kDevTimeoutEmpty = 2,   // the producer waited for a stage that was never released
+  kDevBadIndex = 3,       // KVSWAP_CHECK_INDICES: a group index or count out of range was skipped or clamped
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {

@@ -415,7 +415,6 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
   constexpr uint32_t HALFB = kTok * ROWB;                      // K (or V) part of a stage
   constexpr uint32_t STAGEB = 2 * HALFB;
   constexpr uint32_t kFull = 0xffffffffu;
-  (void)err;                                                   // no wait in this kernel can run out
 
   extern __shared__ unsigned char smem_raw[];
   Control* ctl = reinterpret_cast<Control*>(smem_raw);
@@ -454,7 +453,18 @@ sparse_decode_splitk_kernel(Problem p, const Q_T* __restrict__ q, const KV_T* __
     src.v_begin = min(total, per_split * split);
     src.v_end = min(total, src.v_begin + per_split);
   }
-  const int n_sel = max(0, min(n_selected[int64_t(b) * p.S + srow], p.M));
+  const int n_sel_given = n_selected[int64_t(b) * p.S + srow];
+  const int n_sel = max(0, min(n_sel_given, p.M));
+  // KVSWAP_CHECK_INDICES: the first split of each list looks it over once, ahead of the loop (which skips what
+  // is out of range either way), and records what it finds.  (No wait in this kernel can run out: err serves this only.)
+  if ((p.flags & KVSWAP_CHECK_INDICES) != 0 && err != nullptr && split == 0) {
+    bool bad = n_sel != n_sel_given;
+    for (int i = threadIdx.x; i < n_sel; i += kThreads) {
+      const int j = src.idx[i];
+      bad = bad || (j != -1 && (j < 0 || j >= p.NG));
+    }
+    if (bad) atomicExch(err, kDevBadIndex);
+  }
   const int n_chunks = (src.v_end - src.v_begin + kTok - 1) / kTok;
   const int my_chunks = (n_chunks > warp) ? (n_chunks - warp + kWarps - 1) / kWarps : 0;   // of this warp
 

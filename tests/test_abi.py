@@ -88,7 +88,8 @@ def test_validation_status_codes(lib):
     assert lib.kvswap_validate_shape(None) == 1
     assert kv.kvswap_validate_shape(good_shape(flags=kv.KVSWAP_INPUTS_SETTLED)) == 0
     assert kv.kvswap_validate_shape(good_shape(flags=kv.KVSWAP_SCORE_SOFTMAX | kv.KVSWAP_INPUTS_SETTLED)) == 0
-    assert kv.kvswap_validate_shape(good_shape(flags=4)) == 2          # unknown flag bit
+    assert kv.kvswap_validate_shape(good_shape(flags=kv.KVSWAP_CHECK_INDICES)) == 0
+    assert kv.kvswap_validate_shape(good_shape(flags=8)) == 2          # unknown flag bit
 
 
 def test_entry_points_reject_null_and_small_workspace_without_touching_the_gpu(lib):

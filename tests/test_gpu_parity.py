@@ -273,6 +273,22 @@ def test_sparse_decode_accepts_any_valid_index_list():
     keep = np.delete(base, [3, 7], axis=2)
     out_o, _ = O.attend(li.q, li.K, li.V, keep, 4)
     assert np.abs(out - out_o).max() <= 1e-5
+    assert kv.kvswap_read_device_status(dl.ws) == 0                           # skipped silently ...
+    # ... unless the caller asks for a record: same output, and the status word says what was met
+    checking = dl.shape.with_flags(kv.KVSWAP_CHECK_INDICES)
+    out_c = torch.full_like(dl.out, float("nan"))
+    kv.kvswap_sparse_decode(checking, dl.q, dl.K, dl.V, dl.idx, dl.nsel, out_c, None, dl.ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_c.cpu().numpy(), out)
+    assert kv.kvswap_read_device_status(dl.ws) == 8 and "index" in kv.status_string(8)
+    kv.kvswap_workspace_init(dl.ws)
+    dl.set_selection(base)                                                    # a valid list leaves the word alone
+    kv.kvswap_sparse_decode(checking, dl.q, dl.K, dl.V, dl.idx, dl.nsel, out_c, None, dl.ws)
+    assert kv.kvswap_read_device_status(dl.ws) == 0
+    dl.nsel.fill_(dl.shape.top_k + 3)                                         # a count beyond M is clamped, and recorded
+    kv.kvswap_sparse_decode(checking, dl.q, dl.K, dl.V, dl.idx, dl.nsel, out_c, None, dl.ws)
+    assert kv.kvswap_read_device_status(dl.ws) == 8
+    kv.kvswap_workspace_init(dl.ws)
 
 
 @pytest.mark.parametrize("which", ["cfg1", "cfg3-small", "cfg4-small", "cfg5-small"])
